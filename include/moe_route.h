@@ -1,0 +1,163 @@
+/*
+ * moe_route.h -- C ABI of the B200 (sm_100a) MoE routing and load-control
+ * library for ID Balancing (arXiv 2609.39137).
+ *
+ * One context routes the tokens of L independent router layers per step and
+ * runs one bias-controller step for all of them:
+ *
+ *   logits z = W_r x                         Section 2.2
+ *   score  s = sigmoid(z)                    Section 2.2 / Section 4.3
+ *   select T(x) = TopK_i (s_i + b_i)         Eq. 2
+ *   gates  w_k = s_k / sum_{j in T(x)} s_j   sentence after Eq. 2 (no bias)
+ *   loads  n_i += #tokens assigned to i      Algorithm 1 line 4
+ *   error  e_i = (nbar - n_i) / nbar         Eq. 3, Algorithm 1 lines 5-7
+ *   bias   ID update + centring              Algorithm 1 lines 8-13, Eq. 9-12
+ *          fixed-step integral (DeepSeek)    Eq. 5
+ *          quantile target (proportional)    Eq. 6-7, EMA variant Section 3
+ *   MaxVio / MinVio                          Eq. 13
+ *
+ * Conventions
+ *   - Every tensor pointer is DEVICE memory owned by the caller unless the
+ *     parameter name ends in `_host`.  The library allocates no device memory:
+ *     its state lives in the caller-provided workspace.  Pointers are borrowed
+ *     only for the duration of the enqueued work.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = default stream) and is asynchronous unless stated otherwise.
+ *   - Every call returns a MOE_* status; 0 is success.  Argument errors are
+ *     found on the host before anything is launched.  Nothing throws, aborts
+ *     or prints.  Device-side problems (a bounded wait that expired) are
+ *     sticky in the workspace and reported by moe_route_poll.
+ *   - A context is thread-compatible: one thread at a time per context.
+ *   - Layouts are row-major with the last index fastest:
+ *       x        [L][T][H]  bf16        hidden states, T = num_tokens
+ *       w        [L][E][H]  bf16        router weights W_r (one row per expert)
+ *       topk_idx [L][T][K]  int32       selected experts, by descending biased
+ *                                        score, equal scores by ascending index
+ *       topk_gate[L][T][K]  float32     combination weights in the same order
+ *       logits   [L][T][E]  float32     optional dump of z
+ *       alpha    [L][T]     float32     optional (K+1)-th largest biased score
+ *       loads    [L][E]     int32
+ *       bias, e_prev [L][E] float32
+ */
+#ifndef MOE_ROUTE_H_
+#define MOE_ROUTE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_route_ctx moe_route_ctx; /* opaque, host memory, library-owned */
+
+enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = 1,
+  MOE_ERR_UNSUPPORTED = 2,
+  MOE_ERR_CUDA = 3,
+  MOE_ERR_STATE = 4,      /* e.g. controller update with no tokens routed */
+  MOE_ERR_WORKSPACE = 5,  /* workspace too small or misaligned */
+  MOE_ERR_TIMEOUT = 6     /* a bounded device-side wait expired */
+};
+
+enum {
+  MOE_CTRL_ID = 0,         /* Algorithm 1 */
+  MOE_CTRL_FIXED_STEP = 1, /* Eq. 5 */
+  MOE_CTRL_QUANTILE = 2,   /* Eq. 6-7 */
+  MOE_CTRL_FROZEN = 3      /* bias never changes (continued pretraining /
+                              inference, Section 4.1); loads and metrics only */
+};
+
+typedef struct {
+  int32_t struct_size;  /* = sizeof(moe_route_config) */
+  int32_t num_layers;   /* L >= 1 */
+  int32_t num_experts;  /* E, multiple of 8, K < E <= 1024 (768 is the tuned case) */
+  int32_t top_k;        /* K in 1..16 */
+  int32_t hidden;       /* H, multiple of 8 */
+  int32_t max_tokens;   /* upper bound on num_tokens per call */
+  int32_t controller;   /* MOE_CTRL_* */
+  float ki, kd;         /* ID gains; paper default 6e-3 each (Section 4) */
+  float eta;            /* fixed-step size; paper default 1e-3 (Section 4.1) */
+  float qb_ema_rho;     /* 0 <= rho < 1; 0 = plain Quantile Balancing */
+  int32_t center;       /* zero-mean centring after the update: 1 on, 0 off,
+                           -1 = per-controller default (ID on, others off) */
+  int32_t spin_limit;   /* iteration bound of every device-side wait; 0 = default */
+  int32_t host_staging; /* 1 = reserve workspace for moe_route_step_host */
+} moe_route_config;
+
+/* Fills *cfg with the paper's defaults (Ki = Kd = 6e-3, eta = 1e-3, rho = 0,
+ * centre = -1, ID controller) for the given shape. */
+void moe_route_default_config(moe_route_config* cfg, int32_t num_layers, int32_t num_experts,
+                              int32_t top_k, int32_t hidden, int32_t max_tokens);
+
+/* Bytes of device workspace a context with this config needs (0 on a bad
+ * config).  The caller allocates it (256-byte aligned) and keeps it alive
+ * until moe_route_destroy. */
+size_t moe_route_workspace_bytes(const moe_route_config* cfg);
+
+/* Creates a context on the current CUDA device.  Clears the workspace (bias,
+ * previous error, load accumulators = 0: Algorithm 1 line 1).  Synchronous. */
+int moe_route_init(const moe_route_config* cfg, void* dev_workspace, size_t workspace_bytes,
+                   moe_route_ctx** out);
+
+/* Routes num_tokens tokens in each of the L layers with the current bias held
+ * fixed (Algorithm 1 line 3) and ADDS the selections to the per-expert load
+ * accumulators (line 4) -- several calls before a controller update are the
+ * microbatch case.  logits_out and alpha_out may be NULL.  With
+ * MOE_CTRL_QUANTILE both must be given (L must be 1); they are read again by
+ * the next moe_controller_update and must stay valid until then. */
+int moe_route_step(moe_route_ctx* ctx, const void* x_bf16, const void* w_bf16, int32_t num_tokens,
+                   int32_t* topk_idx, float* topk_gate, float* logits_out, float* alpha_out,
+                   void* cuda_stream);
+
+/* Same step with HOST buffers (pinned memory recommended): copies x (and w if
+ * w_bf16_host is not NULL; otherwise the weights of the previous call are
+ * reused) to the staging area of the workspace, routes, copies indices and
+ * gates back.  Needs host_staging = 1.  Asynchronous on the stream. */
+int moe_route_step_host(moe_route_ctx* ctx, const void* x_bf16_host, const void* w_bf16_host,
+                        int32_t num_tokens, int32_t* topk_idx_host, float* topk_gate_host,
+                        void* cuda_stream);
+
+/* One controller step for all layers (Algorithm 1 lines 5-13, or Eq. 5, or
+ * Eq. 6-7): consumes the load accumulators, updates bias and previous error,
+ * stores loads / MaxVio / MinVio of the consumed step, zeroes the
+ * accumulators.  A layer whose accumulators sum to zero is left unchanged and
+ * the call reports MOE_ERR_STATE through moe_route_poll. */
+int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream);
+
+/* Copies out the loads and MaxVio/MinVio (Eq. 13) of the most recently
+ * consumed step and the current bias.  Any pointer may be NULL. */
+int moe_load_stats(moe_route_ctx* ctx, int32_t* loads, float* bias, float* maxvio, float* minvio,
+                   void* cuda_stream);
+
+/* Number of open derivative gates (g_i = 1, Eq. 11) per layer in the most
+ * recent ID update: gate_count [L] int32. */
+int moe_gate_stats(moe_route_ctx* ctx, int32_t* gate_count, void* cuda_stream);
+
+/* Load accumulators not yet consumed: read them, or add external counts
+ * (Algorithm 1 line 4: counts are summed over microbatches and the
+ * data-parallel group -- a caller that shards tokens adds its peers' counts). */
+int moe_loads_peek(moe_route_ctx* ctx, int32_t* loads, void* cuda_stream);
+int moe_loads_add(moe_route_ctx* ctx, const int32_t* loads, void* cuda_stream);
+
+/* Controller state (b, e_prev of Algorithm 1) for checkpoint / resume. */
+int moe_state_export(moe_route_ctx* ctx, float* bias, float* e_prev, void* cuda_stream);
+int moe_state_import(moe_route_ctx* ctx, const float* bias, const float* e_prev, void* cuda_stream);
+
+/* Synchronises the stream of the last call and returns the sticky device
+ * status (MOE_OK, MOE_ERR_TIMEOUT, MOE_ERR_STATE, MOE_ERR_CUDA); clears it. */
+int moe_route_poll(moe_route_ctx* ctx);
+
+/* Number of kernels this context has launched so far. */
+int64_t moe_route_launch_count(const moe_route_ctx* ctx);
+
+/* Text of the last error of this context ("" if none); valid until the next call. */
+const char* moe_last_error(const moe_route_ctx* ctx);
+
+int moe_route_destroy(moe_route_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_ROUTE_H_ */

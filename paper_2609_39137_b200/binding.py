@@ -1,0 +1,203 @@
+"""ctypes binding of include/moe_route.h (same names, argument marshalling only).
+
+PyTorch appears only as the owner of device memory and streams: tensors are
+passed as raw device pointers.  There is no CPU fallback: if the CUDA library
+is missing, loading fails with an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoe_route_b200.so")
+
+MOE_OK, MOE_ERR_INVALID_ARG, MOE_ERR_UNSUPPORTED, MOE_ERR_CUDA, MOE_ERR_STATE, MOE_ERR_WORKSPACE, MOE_ERR_TIMEOUT = range(7)
+MOE_CTRL_ID, MOE_CTRL_FIXED_STEP, MOE_CTRL_QUANTILE, MOE_CTRL_FROZEN = range(4)
+CONTROLLERS = {"id": MOE_CTRL_ID, "fixed_step": MOE_CTRL_FIXED_STEP, "quantile": MOE_CTRL_QUANTILE,
+               "frozen": MOE_CTRL_FROZEN}
+
+# every symbol include/moe_route.h declares
+SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_init", "moe_route_step",
+           "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
+           "moe_loads_add", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
+           "moe_last_error", "moe_route_destroy"]
+
+
+class MoeRouteConfig(C.Structure):
+    _fields_ = [("struct_size", C.c_int32), ("num_layers", C.c_int32), ("num_experts", C.c_int32),
+                ("top_k", C.c_int32), ("hidden", C.c_int32), ("max_tokens", C.c_int32), ("controller", C.c_int32),
+                ("ki", C.c_float), ("kd", C.c_float), ("eta", C.c_float), ("qb_ema_rho", C.c_float),
+                ("center", C.c_int32), ("spin_limit", C.c_int32), ("host_staging", C.c_int32)]
+
+
+class MoeRouteError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"moe_route error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load():
+    """Loads libmoe_route_b200.so (built in-tree by `build.py`); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(f"{LIB_PATH} not found: build it with `python -m paper_2609_39137_b200.build` "
+                                "(there is no fallback path)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, cfgp = C.c_void_p, C.c_int32, C.POINTER(MoeRouteConfig)
+    L.moe_route_default_config.argtypes = [cfgp, i32, i32, i32, i32, i32]
+    L.moe_route_default_config.restype = None
+    L.moe_route_workspace_bytes.argtypes = [cfgp]
+    L.moe_route_workspace_bytes.restype = C.c_size_t
+    L.moe_route_init.argtypes = [cfgp, vp, C.c_size_t, C.POINTER(vp)]
+    L.moe_route_step.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    L.moe_route_step_host.argtypes = [vp, vp, vp, i32, vp, vp, vp]
+    L.moe_controller_update.argtypes = [vp, vp]
+    L.moe_load_stats.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.moe_gate_stats.argtypes = [vp, vp, vp]
+    L.moe_loads_peek.argtypes = [vp, vp, vp]
+    L.moe_loads_add.argtypes = [vp, vp, vp]
+    L.moe_state_export.argtypes = [vp, vp, vp, vp]
+    L.moe_state_import.argtypes = [vp, vp, vp, vp]
+    L.moe_route_poll.argtypes = [vp]
+    L.moe_route_launch_count.argtypes = [vp]
+    L.moe_route_launch_count.restype = C.c_int64
+    L.moe_last_error.argtypes = [vp]
+    L.moe_last_error.restype = C.c_char_p
+    L.moe_route_destroy.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def default_config(num_layers, num_experts, top_k, hidden, max_tokens) -> MoeRouteConfig:
+    cfg = MoeRouteConfig()
+    load().moe_route_default_config(C.byref(cfg), num_layers, num_experts, top_k, hidden, max_tokens)
+    return cfg
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Router:
+    """One routing + load-control context (L layers).  Methods mirror the C entry points."""
+
+    def __init__(self, num_layers, num_experts, top_k, hidden, max_tokens, controller="id", ki=None, kd=None,
+                 eta=None, qb_ema_rho=None, center=None, spin_limit=0, host_staging=False, device="cuda"):
+        self.lib = load()
+        cfg = default_config(num_layers, num_experts, top_k, hidden, max_tokens)
+        cfg.controller = CONTROLLERS[controller] if isinstance(controller, str) else int(controller)
+        if ki is not None: cfg.ki = ki
+        if kd is not None: cfg.kd = kd
+        if eta is not None: cfg.eta = eta
+        if qb_ema_rho is not None: cfg.qb_ema_rho = qb_ema_rho
+        if center is not None: cfg.center = int(center)
+        cfg.spin_limit = spin_limit
+        cfg.host_staging = int(bool(host_staging))
+        self.cfg = cfg
+        self.L, self.E, self.K, self.H, self.max_tokens = num_layers, num_experts, top_k, hidden, max_tokens
+        self.device = torch.device(device)
+        nbytes = self.lib.moe_route_workspace_bytes(C.byref(cfg))
+        if nbytes == 0:
+            raise MoeRouteError(MOE_ERR_INVALID_ARG, "invalid configuration")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = self.lib.moe_route_init(C.byref(cfg), _ptr(self.workspace), nbytes, C.byref(h))
+        if rc != MOE_OK:
+            raise MoeRouteError(rc, "moe_route_init failed")
+        self.h = h
+
+    def _check(self, rc):
+        if rc != MOE_OK:
+            raise MoeRouteError(rc, self.lib.moe_last_error(self.h).decode())
+
+    # -- moe_route_step
+    def route_step(self, x, w, topk_idx=None, topk_gate=None, logits_out=None, alpha_out=None):
+        """x [L][T][H] bf16, w [L][E][H] bf16 (device). Returns (topk_idx, topk_gate)."""
+        T = x.shape[-2]
+        assert x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16 and x.is_contiguous() and w.is_contiguous()
+        assert x.numel() == self.L * T * self.H and w.numel() == self.L * self.E * self.H
+        if topk_idx is None:
+            topk_idx = torch.empty(self.L, T, self.K, dtype=torch.int32, device=x.device)
+        if topk_gate is None:
+            topk_gate = torch.empty(self.L, T, self.K, dtype=torch.float32, device=x.device)
+        self._check(self.lib.moe_route_step(self.h, _ptr(x), _ptr(w), T, _ptr(topk_idx), _ptr(topk_gate),
+                                            _ptr(logits_out), _ptr(alpha_out), _stream()))
+        return topk_idx, topk_gate
+
+    # -- moe_route_step_host
+    def route_step_host(self, x_host, w_host, topk_idx_host, topk_gate_host):
+        T = x_host.shape[-2]
+        self._check(self.lib.moe_route_step_host(self.h, _ptr(x_host), _ptr(w_host), T, _ptr(topk_idx_host),
+                                                 _ptr(topk_gate_host), _stream()))
+
+    # -- moe_controller_update
+    def controller_update(self):
+        self._check(self.lib.moe_controller_update(self.h, _stream()))
+
+    # -- moe_load_stats
+    def load_stats(self):
+        dev = self.device
+        loads = torch.empty(self.L, self.E, dtype=torch.int32, device=dev)
+        bias = torch.empty(self.L, self.E, dtype=torch.float32, device=dev)
+        maxvio = torch.empty(self.L, dtype=torch.float32, device=dev)
+        minvio = torch.empty(self.L, dtype=torch.float32, device=dev)
+        self._check(self.lib.moe_load_stats(self.h, _ptr(loads), _ptr(bias), _ptr(maxvio), _ptr(minvio), _stream()))
+        return loads, bias, maxvio, minvio
+
+    def gate_stats(self):
+        g = torch.empty(self.L, dtype=torch.int32, device=self.device)
+        self._check(self.lib.moe_gate_stats(self.h, _ptr(g), _stream()))
+        return g
+
+    def loads_peek(self):
+        loads = torch.empty(self.L, self.E, dtype=torch.int32, device=self.device)
+        self._check(self.lib.moe_loads_peek(self.h, _ptr(loads), _stream()))
+        return loads
+
+    def loads_add(self, loads):
+        assert loads.dtype == torch.int32 and loads.is_contiguous() and loads.numel() == self.L * self.E
+        self._check(self.lib.moe_loads_add(self.h, _ptr(loads), _stream()))
+
+    def state_export(self):
+        bias = torch.empty(self.L, self.E, dtype=torch.float32, device=self.device)
+        e_prev = torch.empty(self.L, self.E, dtype=torch.float32, device=self.device)
+        self._check(self.lib.moe_state_export(self.h, _ptr(bias), _ptr(e_prev), _stream()))
+        return bias, e_prev
+
+    def state_import(self, bias=None, e_prev=None):
+        for t in (bias, e_prev):
+            assert t is None or (t.dtype == torch.float32 and t.is_contiguous() and t.numel() == self.L * self.E)
+        self._check(self.lib.moe_state_import(self.h, _ptr(bias), _ptr(e_prev), _stream()))
+
+    def poll(self, raise_on_error=True):
+        rc = self.lib.moe_route_poll(self.h)
+        if rc != MOE_OK and raise_on_error:
+            raise MoeRouteError(rc, self.lib.moe_last_error(self.h).decode())
+        return rc
+
+    def launch_count(self):
+        return int(self.lib.moe_route_launch_count(self.h))
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.moe_route_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

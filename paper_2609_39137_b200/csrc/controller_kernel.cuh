@@ -1,0 +1,147 @@
+// Bias-controller step for all layers in one launch: one CTA of 1024 threads
+// per layer, thread i owns expert i.
+//   error        e_i = (nbar - n_i) / nbar                    Eq. 3
+//   ID           Algorithm 1 lines 8-13 (Eq. 9-12)
+//   fixed step   b += eta * sign(e)                           Eq. 5
+//   quantile     b = rho * b + (1 - rho) * Q                  Eq. 6-7 + EMA (Section 3)
+//   frozen       b unchanged
+//   metrics      MaxVio, MinVio                               Eq. 13
+// Arithmetic: error and metrics in binary64 rounded once to binary32; the
+// update in binary32 with explicitly rounded operations (nothing contracted);
+// the centring mean is a binary64 pairwise sum over 1024 padded entries with
+// strides 512, 256, ..., 1.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace moe {
+
+constexpr int kCtrlThreads = 1024;
+constexpr int kStatusState = 4;  // = MOE_ERR_STATE
+
+struct CtrlParams {
+  int L, E;
+  int controller;  // MOE_CTRL_*
+  float ki, kd, eta, rho;
+  int center;
+  float* bias;        // [L][E] in/out
+  float* e_prev;      // [L][E] in/out
+  int* loads_acc;     // [L][E] consumed and zeroed
+  int* loads_last;    // [L][E] out
+  float* maxvio;      // [L] out
+  float* minvio;      // [L] out
+  int* gate_count;    // [L] out
+  const float* qb_target;  // [L][E], quantile controller only
+  int* status;
+};
+
+__global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlParams p) {
+  __shared__ double y[kCtrlThreads];
+  __shared__ long long red_sum[32];
+  __shared__ int red_max[32], red_min[32], red_gate[32];
+  __shared__ long long total_s;
+  __shared__ int max_s, min_s;
+
+  const int layer = blockIdx.x;
+  const int i = threadIdx.x;
+  const int lane = i & 31, warp = i >> 5;
+  const bool live = i < p.E;
+  const size_t o = (size_t)layer * p.E + i;
+
+  const int n = live ? p.loads_acc[o] : 0;
+  long long s = n;
+  int mx = live ? n : INT_MIN;
+  int mn = live ? n : INT_MAX;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, d);
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, d));
+  }
+  if (lane == 0) { red_sum[warp] = s; red_max[warp] = mx; red_min[warp] = mn; }
+  __syncthreads();
+  if (warp == 0) {
+    s = red_sum[lane]; mx = red_max[lane]; mn = red_min[lane];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      s += __shfl_xor_sync(0xffffffffu, s, d);
+      mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+      mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, d));
+    }
+    if (lane == 0) { total_s = s; max_s = mx; min_s = mn; }
+  }
+  __syncthreads();
+  const long long total = total_s;
+  if (total <= 0) {
+    // empty batch: the error of Eq. 3 is undefined; leave the layer untouched
+    if (i == 0) atomicCAS(p.status, 0, kStatusState);
+    return;
+  }
+  const double nbar = __ddiv_rn((double)total, (double)p.E);
+  const float e = live ? (float)__ddiv_rn(__dsub_rn(nbar, (double)n), nbar) : 0.0f;
+
+  float b = live ? p.bias[o] : 0.0f;
+  const float ep = live ? p.e_prev[o] : 0.0f;
+  int gate = 0;
+  if (p.controller == 0) {                       // ID Balancing
+    const float de = __fsub_rn(e, ep);
+    gate = ((ep > 0.0f && de > 0.0f) || (ep < 0.0f && de < 0.0f)) ? 1 : 0;
+    const float t1 = __fmul_rn(p.ki, e);
+    const float t2 = gate ? __fmul_rn(p.kd, de) : 0.0f;
+    b = __fadd_rn(__fadd_rn(b, t1), t2);
+  } else if (p.controller == 1) {                // fixed-step integral
+    const float step = (e > 0.0f) ? p.eta : (e < 0.0f) ? -p.eta : 0.0f;
+    b = __fadd_rn(b, step);
+  } else if (p.controller == 2) {                // quantile target (+ EMA)
+    const float q = live ? p.qb_target[o] : 0.0f;
+    if (p.rho == 0.0f) {
+      b = q;
+    } else {
+      const float keep = __fmul_rn(p.rho, b);
+      const float take = __fmul_rn(__fsub_rn(1.0f, p.rho), q);
+      b = __fadd_rn(keep, take);
+    }
+  }
+  if (!live) gate = 0;
+
+  if (p.center) {
+    y[i] = live ? (double)b : 0.0;
+    __syncthreads();
+#pragma unroll 1
+    for (int stride = kCtrlThreads / 2; stride >= 1; stride >>= 1) {
+      // y[i + stride] is not written during this pass, so one barrier suffices
+      if (i < stride) y[i] = __dadd_rn(y[i], y[i + stride]);
+      __syncthreads();
+    }
+    const float mean = (float)__ddiv_rn(y[0], (double)p.E);
+    b = __fsub_rn(b, mean);
+  }
+
+  int gsum = gate;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) gsum += __shfl_xor_sync(0xffffffffu, gsum, d);
+  if (lane == 0) red_gate[warp] = gsum;
+  __syncthreads();
+
+  if (live) {
+    p.bias[o] = b;
+    p.e_prev[o] = e;
+    p.loads_last[o] = n;
+    p.loads_acc[o] = 0;
+  }
+  if (i == 0) {
+    int gtot = 0;
+    for (int w = 0; w < kCtrlThreads / 32; ++w) gtot += red_gate[w];
+    p.gate_count[layer] = gtot;
+    p.maxvio[layer] = (float)__ddiv_rn(__dsub_rn((double)max_s, nbar), nbar);
+    p.minvio[layer] = (float)__ddiv_rn(__dsub_rn(nbar, (double)min_s), nbar);
+  }
+}
+
+// loads_acc[i] += add[i]
+__global__ void loads_add_kernel(int* acc, const int* add, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) acc[i] += add[i];
+}
+
+}  // namespace moe

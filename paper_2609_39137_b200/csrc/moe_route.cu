@@ -1,0 +1,452 @@
+// Host side of the C ABI declared in include/moe_route.h: argument checks,
+// workspace layout, TMA descriptors, kernel launches.  No device memory is
+// allocated here; all state lives in the caller's workspace.
+#include "../../include/moe_route.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "controller_kernel.cuh"
+#include "quantile_kernel.cuh"
+#include "route_kernel.cuh"
+
+namespace {
+
+using namespace moe;
+
+constexpr size_t kAlign = 256;
+constexpr size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+  size_t status, bias, e_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
+  size_t qb_target, qb_hist, qb_prefix, qb_rank;
+  size_t state_end;  // everything before this is cleared at init
+  size_t stage_x, stage_w, stage_idx, stage_gate;
+  size_t total;
+};
+
+Layout make_layout(const moe_route_config& c) {
+  Layout l{};
+  size_t o = 0;
+  const size_t LE = (size_t)c.num_layers * c.num_experts;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  l.status = take(64);
+  l.bias = take(LE * 4);
+  l.e_prev = take(LE * 4);
+  l.loads_acc = take(LE * 4);
+  l.loads_last = take(LE * 4);
+  l.maxvio = take((size_t)c.num_layers * 4);
+  l.minvio = take((size_t)c.num_layers * 4);
+  l.gate_count = take((size_t)c.num_layers * 4);
+  l.qb_target = take(LE * 4);
+  if (c.controller == MOE_CTRL_QUANTILE) {
+    l.qb_hist = take((size_t)c.num_experts * 256 * 4);
+    l.qb_prefix = take((size_t)c.num_experts * 4);
+    l.qb_rank = take((size_t)c.num_experts * 4);
+  }
+  l.state_end = o;
+  if (c.host_staging) {
+    const size_t LT = (size_t)c.num_layers * c.max_tokens;
+    l.stage_x = take(LT * c.hidden * 2);
+    l.stage_w = take(LE * c.hidden * 2);
+    l.stage_idx = take(LT * c.top_k * 4);
+    l.stage_gate = take(LT * c.top_k * 4);
+  }
+  l.total = o;
+  return l;
+}
+
+bool config_ok(const moe_route_config* c) {
+  if (!c || c->struct_size != (int32_t)sizeof(moe_route_config)) return false;
+  if (c->num_layers < 1 || c->num_layers > 65535) return false;
+  if (c->num_experts < 8 || c->num_experts > kMaxE || (c->num_experts % 8) != 0) return false;
+  if (c->top_k < 1 || c->top_k > 16 || c->top_k >= c->num_experts) return false;
+  if (c->hidden < 8 || (c->hidden % 8) != 0) return false;
+  if (c->max_tokens < 1) return false;
+  if (c->controller < MOE_CTRL_ID || c->controller > MOE_CTRL_FROZEN) return false;
+  if (!(c->ki >= 0.0f) || !(c->kd >= 0.0f) || !(c->eta >= 0.0f)) return false;
+  if (!(c->qb_ema_rho >= 0.0f) || !(c->qb_ema_rho < 1.0f)) return false;
+  if (c->center < -1 || c->center > 1) return false;
+  if (c->spin_limit < 0) return false;
+  if (c->controller == MOE_CTRL_QUANTILE && c->num_layers != 1) return false;
+  return true;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct moe_route_ctx {
+  moe_route_config cfg;
+  Layout lay;
+  uint8_t* ws;
+  int device;
+  int num_sms;
+  int center_on;
+  EncodeTiledFn encode;
+  cudaStream_t last_stream;
+  int64_t launches;
+  // cached TMA descriptors
+  const void* map_x_ptr;
+  const void* map_w_ptr;
+  int map_tokens;
+  CUtensorMap tm_x, tm_w;
+  // quantile controller: dump of the last routing step
+  const float* qb_logits;
+  const float* qb_alpha;
+  int qb_tokens;
+  bool staged_w;
+  char err[256];
+};
+
+namespace {
+
+int fail(moe_route_ctx* ctx, int code, const char* fmt, ...) {
+  if (ctx) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+int cuda_fail(moe_route_ctx* ctx, cudaError_t e, const char* what) {
+  return fail(ctx, MOE_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+template <typename T>
+T* at(moe_route_ctx* ctx, size_t off) { return reinterpret_cast<T*>(ctx->ws + off); }
+
+int* status_ptr(moe_route_ctx* ctx) { return at<int>(ctx, ctx->lay.status); }
+
+// 3-D bf16 tensor map: dims (inner, rows, layers), box (64, box_rows, 1), 128-byte swizzle,
+// out-of-range elements read as zero.
+int encode_map(moe_route_ctx* ctx, CUtensorMap* out, const void* base, uint64_t inner, uint64_t rows,
+               uint64_t layers, uint32_t box_rows) {
+  cuuint64_t dims[3] = {inner, rows, layers};
+  cuuint64_t strides[2] = {inner * 2, inner * rows * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kBK, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  return MOE_OK;
+}
+
+template <int KL>
+int launch_route(moe_route_ctx* ctx, const RouteParams& rp, int grid, cudaStream_t st) {
+  static bool attr_set[64] = {};
+  const size_t smem = route_smem_bytes<KL>();
+  if (!attr_set[ctx->device & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(route_step_kernel<KL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(route_step_kernel)");
+    attr_set[ctx->device & 63] = true;
+  }
+  route_step_kernel<KL><<<grid, kRouteThreads, smem, st>>>(ctx->tm_x, ctx->tm_w, rp);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "route_step_kernel launch");
+  ctx->launches += 1;
+  return MOE_OK;
+}
+
+int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, int32_t* idx, float* gate,
+                 float* logits, float* alpha, cudaStream_t st) {
+  const moe_route_config& c = ctx->cfg;
+  if (ctx->map_x_ptr != x || ctx->map_w_ptr != w || ctx->map_tokens != T) {
+    if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(w) & 15))
+      return fail(ctx, MOE_ERR_INVALID_ARG, "x and w must be 16-byte aligned");
+    int rc = encode_map(ctx, &ctx->tm_x, x, c.hidden, T, c.num_layers, kBM);
+    if (rc) return rc;
+    rc = encode_map(ctx, &ctx->tm_w, w, c.hidden, c.num_experts, c.num_layers, kBN);
+    if (rc) return rc;
+    ctx->map_x_ptr = x; ctx->map_w_ptr = w; ctx->map_tokens = T;
+  }
+  RouteParams rp{};
+  rp.L = c.num_layers; rp.T = T; rp.H = c.hidden; rp.E = c.num_experts; rp.K = c.top_k;
+  rp.tiles_per_layer = (T + kBM - 1) / kBM;
+  rp.num_items = rp.tiles_per_layer * c.num_layers;
+  rp.num_kblocks = (c.hidden + kBK - 1) / kBK;
+  rp.num_chunks = (c.num_experts + kBN - 1) / kBN;
+  rp.bias = at<float>(ctx, ctx->lay.bias);
+  rp.loads = at<int>(ctx, ctx->lay.loads_acc);
+  rp.topk_idx = idx; rp.topk_gate = gate; rp.logits_out = logits; rp.alpha_out = alpha;
+  rp.status = status_ptr(ctx);
+  rp.spin_limit = c.spin_limit > 0 ? (uint32_t)c.spin_limit : 0x7fffffffu;
+  const int grid = rp.num_items < ctx->num_sms ? rp.num_items : ctx->num_sms;
+  const int need = c.top_k + (alpha ? 1 : 0);
+  if (need <= 3) return launch_route<3>(ctx, rp, grid, st);
+  if (need <= 5) return launch_route<5>(ctx, rp, grid, st);
+  if (need <= 8) return launch_route<8>(ctx, rp, grid, st);
+  if (need <= 10) return launch_route<10>(ctx, rp, grid, st);
+  return launch_route<17>(ctx, rp, grid, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+void moe_route_default_config(moe_route_config* cfg, int32_t num_layers, int32_t num_experts, int32_t top_k,
+                              int32_t hidden, int32_t max_tokens) {
+  if (!cfg) return;
+  memset(cfg, 0, sizeof *cfg);
+  cfg->struct_size = (int32_t)sizeof *cfg;
+  cfg->num_layers = num_layers;
+  cfg->num_experts = num_experts;
+  cfg->top_k = top_k;
+  cfg->hidden = hidden;
+  cfg->max_tokens = max_tokens;
+  cfg->controller = MOE_CTRL_ID;
+  cfg->ki = 6e-3f;
+  cfg->kd = 6e-3f;
+  cfg->eta = 1e-3f;
+  cfg->qb_ema_rho = 0.0f;
+  cfg->center = -1;
+  cfg->spin_limit = 0;
+  cfg->host_staging = 0;
+}
+
+size_t moe_route_workspace_bytes(const moe_route_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return make_layout(*cfg).total;
+}
+
+int moe_route_init(const moe_route_config* cfg, void* dev_workspace, size_t workspace_bytes, moe_route_ctx** out) {
+  if (!out) return MOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(cfg)) return MOE_ERR_INVALID_ARG;
+  const Layout lay = make_layout(*cfg);
+  if (!dev_workspace || workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(dev_workspace) % kAlign) != 0)
+    return MOE_ERR_WORKSPACE;
+  moe_route_ctx* ctx = new (std::nothrow) moe_route_ctx();
+  if (!ctx) return MOE_ERR_CUDA;
+  ctx->cfg = *cfg;
+  ctx->lay = lay;
+  ctx->ws = static_cast<uint8_t*>(dev_workspace);
+  ctx->center_on = cfg->center >= 0 ? cfg->center : (cfg->controller == MOE_CTRL_ID ? 1 : 0);
+  if (cfg->controller == MOE_CTRL_FROZEN) ctx->center_on = 0;
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
+  int major = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, ctx->device);
+  if (e != cudaSuccess) { delete ctx; return MOE_ERR_CUDA; }
+  if (major != 10) { delete ctx; return MOE_ERR_UNSUPPORTED; }   // sm_100a code only
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) { delete ctx; return MOE_ERR_CUDA; }
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  e = cudaMemset(dev_workspace, 0, lay.state_end);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) { delete ctx; return MOE_ERR_CUDA; }
+  *out = ctx;
+  return MOE_OK;
+}
+
+int moe_route_step(moe_route_ctx* ctx, const void* x_bf16, const void* w_bf16, int32_t num_tokens,
+                   int32_t* topk_idx, float* topk_gate, float* logits_out, float* alpha_out, void* cuda_stream) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (!x_bf16 || !w_bf16 || !topk_idx || !topk_gate) return fail(ctx, MOE_ERR_INVALID_ARG, "null tensor pointer");
+  if (num_tokens < 1 || num_tokens > ctx->cfg.max_tokens)
+    return fail(ctx, MOE_ERR_INVALID_ARG, "num_tokens %d outside [1, %d]", num_tokens, ctx->cfg.max_tokens);
+  if (ctx->cfg.controller == MOE_CTRL_QUANTILE && (!logits_out || !alpha_out))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "the quantile controller needs logits_out and alpha_out");
+  if (ctx->cfg.controller == MOE_CTRL_QUANTILE && ctx->qb_logits != nullptr) {
+    // Eq. 7 ranks the margins of ONE score matrix; a second routing call
+    // before the update would need a merged dump.
+    return fail(ctx, MOE_ERR_UNSUPPORTED, "quantile controller: one routing step per controller update");
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  int rc = route_device(ctx, x_bf16, w_bf16, num_tokens, topk_idx, topk_gate, logits_out, alpha_out, st);
+  if (rc == MOE_OK && ctx->cfg.controller == MOE_CTRL_QUANTILE) {
+    ctx->qb_logits = logits_out; ctx->qb_alpha = alpha_out; ctx->qb_tokens = num_tokens;
+  }
+  return rc;
+}
+
+int moe_route_step_host(moe_route_ctx* ctx, const void* x_bf16_host, const void* w_bf16_host, int32_t num_tokens,
+                        int32_t* topk_idx_host, float* topk_gate_host, void* cuda_stream) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  const moe_route_config& c = ctx->cfg;
+  if (!c.host_staging) return fail(ctx, MOE_ERR_STATE, "context was created without host_staging");
+  if (c.controller == MOE_CTRL_QUANTILE) return fail(ctx, MOE_ERR_UNSUPPORTED, "host step: no quantile controller");
+  if (!x_bf16_host || !topk_idx_host || !topk_gate_host) return fail(ctx, MOE_ERR_INVALID_ARG, "null host pointer");
+  if (!w_bf16_host && !ctx->staged_w) return fail(ctx, MOE_ERR_STATE, "no router weights staged yet");
+  if (num_tokens < 1 || num_tokens > c.max_tokens) return fail(ctx, MOE_ERR_INVALID_ARG, "num_tokens out of range");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  const size_t LT = (size_t)c.num_layers * num_tokens;
+  cudaError_t e = cudaMemcpyAsync(ctx->ws + ctx->lay.stage_x, x_bf16_host, LT * c.hidden * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && w_bf16_host) {
+    e = cudaMemcpyAsync(ctx->ws + ctx->lay.stage_w, w_bf16_host, (size_t)c.num_layers * c.num_experts * c.hidden * 2,
+                        cudaMemcpyHostToDevice, st);
+    ctx->staged_w = true;
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
+  int rc = route_device(ctx, ctx->ws + ctx->lay.stage_x, ctx->ws + ctx->lay.stage_w, num_tokens,
+                        at<int32_t>(ctx, ctx->lay.stage_idx), at<float>(ctx, ctx->lay.stage_gate), nullptr, nullptr, st);
+  if (rc) return rc;
+  e = cudaMemcpyAsync(topk_idx_host, ctx->ws + ctx->lay.stage_idx, LT * c.top_k * 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(topk_gate_host, ctx->ws + ctx->lay.stage_gate, LT * c.top_k * 4, cudaMemcpyDeviceToHost, st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "device to host copy");
+  return MOE_OK;
+}
+
+int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  const moe_route_config& c = ctx->cfg;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  if (c.controller == MOE_CTRL_QUANTILE) {
+    if (!ctx->qb_logits) return fail(ctx, MOE_ERR_STATE, "quantile controller: no routing step since the last update");
+    QbParams q{};
+    q.logits = ctx->qb_logits; q.alpha = ctx->qb_alpha; q.m = ctx->qb_tokens; q.E = c.num_experts; q.K = c.top_k;
+    q.hist = at<uint32_t>(ctx, ctx->lay.qb_hist);
+    q.prefix = at<uint32_t>(ctx, ctx->lay.qb_prefix);
+    q.rank = at<uint32_t>(ctx, ctx->lay.qb_rank);
+    q.target = at<float>(ctx, ctx->lay.qb_target);
+    qb_init_kernel<<<64, 256, 0, st>>>(q);
+    const int col_groups = (c.num_experts + kQbCols - 1) / kQbCols;
+    int splits = (2 * ctx->num_sms + col_groups - 1) / col_groups;
+    const int max_splits = (q.m + 63) / 64;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    for (int pass = 0; pass < 4; ++pass) {
+      qb_hist_kernel<<<dim3(col_groups, splits), kQbThreads, 0, st>>>(q, pass);
+      qb_scan_kernel<<<(c.num_experts * 32 + 255) / 256, 256, 0, st>>>(q, pass);
+    }
+    ctx->launches += 9;
+    ctx->qb_logits = nullptr;
+  }
+  CtrlParams p{};
+  p.L = c.num_layers; p.E = c.num_experts; p.controller = c.controller;
+  p.ki = c.ki; p.kd = c.kd; p.eta = c.eta; p.rho = c.qb_ema_rho; p.center = ctx->center_on;
+  p.bias = at<float>(ctx, ctx->lay.bias);
+  p.e_prev = at<float>(ctx, ctx->lay.e_prev);
+  p.loads_acc = at<int>(ctx, ctx->lay.loads_acc);
+  p.loads_last = at<int>(ctx, ctx->lay.loads_last);
+  p.maxvio = at<float>(ctx, ctx->lay.maxvio);
+  p.minvio = at<float>(ctx, ctx->lay.minvio);
+  p.gate_count = at<int>(ctx, ctx->lay.gate_count);
+  p.qb_target = at<float>(ctx, ctx->lay.qb_target);
+  p.status = status_ptr(ctx);
+  controller_kernel<<<c.num_layers, kCtrlThreads, 0, st>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "controller_kernel launch");
+  ctx->launches += 1;
+  return MOE_OK;
+}
+
+static int copy_out(moe_route_ctx* ctx, void* dst, size_t off, size_t bytes, cudaStream_t st) {
+  if (!dst) return MOE_OK;
+  cudaError_t e = cudaMemcpyAsync(dst, ctx->ws + off, bytes, cudaMemcpyDeviceToDevice, st);
+  return e == cudaSuccess ? MOE_OK : cuda_fail(ctx, e, "device copy");
+}
+
+int moe_load_stats(moe_route_ctx* ctx, int32_t* loads, float* bias, float* maxvio, float* minvio, void* cuda_stream) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  const size_t LE = (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4, Lb = (size_t)ctx->cfg.num_layers * 4;
+  int rc = copy_out(ctx, loads, ctx->lay.loads_last, LE, st);
+  if (!rc) rc = copy_out(ctx, bias, ctx->lay.bias, LE, st);
+  if (!rc) rc = copy_out(ctx, maxvio, ctx->lay.maxvio, Lb, st);
+  if (!rc) rc = copy_out(ctx, minvio, ctx->lay.minvio, Lb, st);
+  return rc;
+}
+
+int moe_gate_stats(moe_route_ctx* ctx, int32_t* gate_count, void* cuda_stream) {
+  if (!ctx || !gate_count) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  return copy_out(ctx, gate_count, ctx->lay.gate_count, (size_t)ctx->cfg.num_layers * 4, st);
+}
+
+int moe_loads_peek(moe_route_ctx* ctx, int32_t* loads, void* cuda_stream) {
+  if (!ctx || !loads) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  return copy_out(ctx, loads, ctx->lay.loads_acc, (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4, st);
+}
+
+int moe_loads_add(moe_route_ctx* ctx, const int32_t* loads, void* cuda_stream) {
+  if (!ctx || !loads) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  const int n = ctx->cfg.num_layers * ctx->cfg.num_experts;
+  loads_add_kernel<<<(n + 255) / 256, 256, 0, st>>>(at<int>(ctx, ctx->lay.loads_acc), loads, n);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "loads_add_kernel launch");
+  ctx->launches += 1;
+  return MOE_OK;
+}
+
+int moe_state_export(moe_route_ctx* ctx, float* bias, float* e_prev, void* cuda_stream) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  const size_t LE = (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4;
+  int rc = copy_out(ctx, bias, ctx->lay.bias, LE, st);
+  if (!rc) rc = copy_out(ctx, e_prev, ctx->lay.e_prev, LE, st);
+  return rc;
+}
+
+int moe_state_import(moe_route_ctx* ctx, const float* bias, const float* e_prev, void* cuda_stream) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  const size_t LE = (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4;
+  cudaError_t e = cudaSuccess;
+  if (bias) e = cudaMemcpyAsync(ctx->ws + ctx->lay.bias, bias, LE, cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess && e_prev) e = cudaMemcpyAsync(ctx->ws + ctx->lay.e_prev, e_prev, LE, cudaMemcpyDeviceToDevice, st);
+  return e == cudaSuccess ? MOE_OK : cuda_fail(ctx, e, "device copy");
+}
+
+int moe_route_poll(moe_route_ctx* ctx) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  cudaError_t e = cudaStreamSynchronize(ctx->last_stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamSynchronize");
+  int st[2] = {0, 0};
+  e = cudaMemcpy(st, status_ptr(ctx), sizeof st, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "status read");
+  if (st[0] != MOE_OK) {
+    cudaMemset(status_ptr(ctx), 0, sizeof st);
+    if (st[0] == MOE_ERR_TIMEOUT)
+      return fail(ctx, MOE_ERR_TIMEOUT, "a bounded device-side wait expired (wait id %d)", st[1]);
+    if (st[0] == MOE_ERR_STATE)
+      return fail(ctx, MOE_ERR_STATE, "controller update on a layer with no routed tokens");
+    return fail(ctx, st[0], "device status %d", st[0]);
+  }
+  return MOE_OK;
+}
+
+int64_t moe_route_launch_count(const moe_route_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* moe_last_error(const moe_route_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+int moe_route_destroy(moe_route_ctx* ctx) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  delete ctx;
+  return MOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,132 @@
+// Quantile Balancing target (Eq. 6-7): for every expert j the r-th smallest
+// margin d_ij = s_ij - alpha_i over the m tokens of the step, Q_j = -d, with
+// the nearest-rank position r = m - floor(m K / E) (no interpolation).
+//
+// Exact selection by a most-significant-digit radix select over the
+// order-preserving 32-bit image of the margin: four passes of 8 bits.  Each
+// pass streams the dumped logits once (HBM-bound, coalesced: a warp reads 32
+// consecutive experts of one token), recomputes the score, and counts -- per
+// expert -- the margins that still match the digits fixed so far, in a
+// shared-memory histogram that is flushed to the global scratch histogram with
+// one atomic per non-empty bin per CTA.  A small scan kernel then fixes the
+// next digit per expert, updates the remaining rank and clears the histogram.
+//
+// Scratch per context: hist [E][256] u32, prefix [E] u32, rank [E] u32.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "route_math.cuh"
+
+namespace moe {
+
+constexpr int kQbCols = 32;       // experts per CTA (one per lane)
+constexpr int kQbThreads = 256;   // 8 warps, each takes every 8th row of the CTA's row range
+
+struct QbParams {
+  const float* logits;  // [m][E]
+  const float* alpha;   // [m]
+  int m, E, K;
+  uint32_t* hist;       // [E][256], zero on entry of every histogram pass
+  uint32_t* prefix;     // [E] digits fixed so far (high bits)
+  uint32_t* rank;       // [E] remaining 1-based rank inside the matching set
+  float* target;        // [E] out: Q_j
+};
+
+// Monotone map float -> uint32 (a < b as floats  <=>  key(a) < key(b)); -0 is
+// canonicalised to +0 first so equal values get equal keys.
+__device__ __forceinline__ uint32_t margin_key(float d) {
+  d = __fadd_rn(d, 0.0f);
+  const uint32_t u = __float_as_uint(d);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float margin_from_key(uint32_t k) {
+  const uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+  return __uint_as_float(u);
+}
+
+__global__ void qb_init_kernel(QbParams p) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < p.E) {
+    long long r = (long long)p.m - ((long long)p.m * p.K) / p.E;
+    if (r < 1) r = 1;
+    if (r > p.m) r = p.m;
+    p.prefix[j] = 0u;
+    p.rank[j] = (uint32_t)r;
+  }
+  for (int i = j; i < p.E * 256; i += gridDim.x * blockDim.x) p.hist[i] = 0u;
+}
+
+// pass = 0..3, most significant byte first.  grid = (ceil(E/32), row_splits)
+__global__ void __launch_bounds__(kQbThreads) qb_hist_kernel(QbParams p, int pass) {
+  __shared__ uint32_t h[256 * kQbCols];  // [bin][col]: lanes hit distinct banks
+  for (int i = threadIdx.x; i < 256 * kQbCols; i += kQbThreads) h[i] = 0u;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int col = blockIdx.x * kQbCols + lane;
+  const bool live = col < p.E;
+  const int shift = 24 - 8 * pass;
+  const uint32_t pre = live ? p.prefix[col] : 0u;
+  const int rows_per = (p.m + gridDim.y - 1) / gridDim.y;
+  const int r0 = blockIdx.y * rows_per;
+  const int r1 = min(p.m, r0 + rows_per);
+  for (int i = r0 + warp; i < r1; i += kQbThreads / 32) {
+    if (live) {
+      const float s = sigmoid_score(p.logits[(size_t)i * p.E + col]);
+      const uint32_t key = margin_key(__fsub_rn(s, p.alpha[i]));
+      const bool match = (pass == 0) || (((key ^ pre) >> (shift + 8)) == 0u);
+      if (match) atomicAdd(&h[((key >> shift) & 255u) * kQbCols + lane], 1u);
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < 256 * kQbCols; i += kQbThreads) {
+    const int c = blockIdx.x * kQbCols + (i % kQbCols);
+    const uint32_t cnt = h[i];
+    if (cnt != 0u && c < p.E) atomicAdd(&p.hist[(size_t)c * 256 + i / kQbCols], cnt);
+  }
+}
+
+// One warp per expert: find the bin holding the remaining rank, fix that
+// digit, clear the histogram; after the last pass emit Q_j = -margin.
+__global__ void qb_scan_kernel(QbParams p, int pass) {
+  const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (j >= p.E) return;
+  uint32_t* hj = p.hist + (size_t)j * 256;
+  uint32_t c[8];
+  uint32_t mine = 0;
+#pragma unroll
+  for (int t = 0; t < 8; ++t) { c[t] = hj[lane * 8 + t]; mine += c[t]; }
+  uint32_t incl = mine;  // inclusive prefix sum over lanes
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  const uint32_t rank = p.rank[j];
+  const uint32_t excl = incl - mine;
+  const bool holder = (rank > excl) && (rank <= incl);   // exactly one lane when 1 <= rank <= total
+  uint32_t bin = 0, below = 0;
+  if (holder) {
+    uint32_t run = excl;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if (rank > run && rank <= run + c[t]) { bin = lane * 8 + t; below = run; }
+      run += c[t];
+    }
+  }
+  const uint32_t who = __ballot_sync(0xffffffffu, holder);
+  const int src = who ? (__ffs(who) - 1) : 0;
+  bin = __shfl_sync(0xffffffffu, bin, src);
+  below = __shfl_sync(0xffffffffu, below, src);
+#pragma unroll
+  for (int t = 0; t < 8; ++t) hj[lane * 8 + t] = 0u;
+  if (lane == 0) {
+    const uint32_t pre = p.prefix[j] | (bin << (24 - 8 * pass));
+    p.prefix[j] = pre;
+    p.rank[j] = rank - below;
+    if (pass == 3) p.target[j] = -margin_from_key(pre);
+  }
+}
+
+}  // namespace moe

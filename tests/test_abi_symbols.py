@@ -1,0 +1,56 @@
+"""Host-only checks of the C-ABI library: it loads, exports every symbol the
+header declares, and validates configurations without touching a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2609_39137_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "moe_route.h")).read()
+    declared = set(re.findall(r"\b(moe_[a-z_]+)\s*\(", header))
+    assert declared == set(binding.SYMBOLS), declared ^ set(binding.SYMBOLS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_config_struct_matches_header(lib):
+    cfg = binding.default_config(2, 768, 10, 2048, 16384)
+    assert cfg.struct_size == C.sizeof(binding.MoeRouteConfig) == 14 * 4
+    # paper defaults: Ki = Kd = 6e-3 (Section 4), eta = 1e-3 (Section 4.1), no EMA
+    assert abs(cfg.ki - 6e-3) < 1e-9 and abs(cfg.kd - 6e-3) < 1e-9 and abs(cfg.eta - 1e-3) < 1e-9
+    assert cfg.qb_ema_rho == 0 and cfg.center == -1 and cfg.controller == binding.MOE_CTRL_ID
+
+
+def test_workspace_bytes_and_config_validation(lib):
+    cfg = binding.default_config(48, 768, 10, 2048, 16384)
+    n = lib.moe_route_workspace_bytes(C.byref(cfg))
+    assert n >= 4 * 48 * 768 * 4 and n % 256 == 0
+    cfg.host_staging = 1
+    assert lib.moe_route_workspace_bytes(C.byref(cfg)) > n + 48 * 16384 * 2048 * 2
+    bad = [dict(num_experts=770), dict(num_experts=2048), dict(top_k=0), dict(top_k=17), dict(hidden=100),
+           dict(num_layers=0), dict(max_tokens=0), dict(controller=7), dict(qb_ema_rho=1.0), dict(ki=-1.0),
+           dict(struct_size=8), dict(controller=binding.MOE_CTRL_QUANTILE)]   # quantile needs L == 1
+    for kw in bad:
+        c = binding.default_config(48, 768, 10, 2048, 16384)
+        for k, v in kw.items():
+            setattr(c, k, v)
+        assert lib.moe_route_workspace_bytes(C.byref(c)) == 0, kw
+    h = C.c_void_p()
+    c = binding.default_config(1, 768, 10, 2048, 128)
+    assert lib.moe_route_init(C.byref(c), None, 0, C.byref(h)) == binding.MOE_ERR_WORKSPACE
+    c.top_k = 0
+    assert lib.moe_route_init(C.byref(c), None, 0, C.byref(h)) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_route_poll(None) == binding.MOE_ERR_INVALID_ARG
+    assert lib.moe_controller_update(None, None) == binding.MOE_ERR_INVALID_ARG
