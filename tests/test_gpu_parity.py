@@ -1,0 +1,353 @@
+"""Parity of the CUDA path (called through the C ABI) against the CPU oracle.
+
+Bars: integer results (expert indices, loads) bit-exact; every fp32 output
+bit-exact given the GPU's own fp32 logits (binary32 chain of the oracle);
+logits within 1e-4 of the fp64 definition computed from the bf16 operands;
+expert sets equal wherever the rank-K/rank-K+1 gap is at least 1e-4.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_39137_b200 import binding, synth
+from parity_util import (NEAR_TIE_BUDGET, THREADS, bits, check_definition, check_exact, full_check, np_,
+                         oracle_controller_step, route_once)
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ routing
+@pytest.mark.parametrize("T,H,E,K,L,alpha", [
+    (128, 64, 256, 3, 1, False),      # one tile, one chunk, one k-block
+    (128, 256, 768, 3, 1, False),     # three chunks
+    (300, 512, 768, 10, 1, False),    # several tiles and a ragged tail
+    (1000, 256, 768, 5, 3, True),     # layers, ragged tail, alpha
+    (513, 192, 768, 10, 2, True),
+    (257, 320, 256, 8, 2, False),     # Top-8-of-256 shape
+    (640, 1024, 768, 3, 1, True),
+])
+def test_route_matches_oracle(T, H, E, K, L, alpha):
+    g = torch.Generator().manual_seed(T + K)
+    bias = torch.randn(L, E, generator=g) * 0.02
+    res = route_once(T, H, E, K, L, bias=bias, seed=T, want_alpha=alpha)
+    full_check(res, K)
+
+
+@pytest.mark.parametrize("T,H,E,K", [
+    (1, 64, 768, 10), (127, 64, 768, 3), (129, 64, 768, 3),     # token tails
+    (64, 8, 768, 5), (200, 72, 768, 5), (96, 136, 768, 10),     # hidden below / not a multiple of 64
+    (256, 64, 8, 3), (256, 64, 40, 16), (256, 128, 1024, 1), (130, 64, 1000, 16),   # expert-count and K extremes
+])
+def test_route_edge_shapes(T, H, E, K):
+    g = torch.Generator().manual_seed(E + K)
+    bias = torch.randn(1, E, generator=g) * 0.05
+    res = route_once(T, H, E, K, 1, bias=bias, seed=E, want_alpha=(K < 16))
+    full_check(res, K)
+
+
+def test_route_operand_layout_one_hot():
+    # one-hot router rows: logit[t][e] = x[t][h(e)] exactly -- exposes any
+    # swizzle / descriptor / transposition error
+    T, H, E, K = 256, 256, 768, 3
+    dev = "cuda"
+    x = torch.randn(1, T, H, device=dev).to(torch.bfloat16)
+    w = torch.zeros(1, E, H, device=dev, dtype=torch.bfloat16)
+    hsel = (torch.arange(E, device=dev) * 7 + 3) % H
+    w[0, torch.arange(E, device=dev), hsel] = 1.0
+    res = route_once(T, H, E, K, x=x, w=w)
+    expect = x[0].float()[:, hsel]
+    np.testing.assert_array_equal(res["logits"][0], np_(expect))
+    full_check(res, K)
+
+
+def test_route_exact_ties_pick_lowest_index():
+    # all-zero hidden states: every logit is 0, every score 0.5 -> with zero
+    # bias the K lowest indices win; with a bias plateau the plateau's lowest
+    T, H, E, K = 200, 64, 768, 10
+    x = torch.zeros(1, T, H, device="cuda", dtype=torch.bfloat16)
+    res = route_once(T, H, E, K, x=x)
+    assert np.all(res["idx"][0] == np.arange(K)[None, :])
+    np.testing.assert_array_equal(res["gate"][0], np.full((T, K), np.float32(1.0) / np.float32(K), np.float32))
+    bias = torch.zeros(1, E)
+    bias[0, 300:320] = 0.25          # plateau straddles two accumulator chunks? no: inside chunk 1, both halves
+    bias[0, 100] = 0.25
+    bias[0, 700] = 0.25
+    res = route_once(T, H, E, K, x=x, bias=bias, want_alpha=True)
+    assert np.all(res["idx"][0] == np.array([100] + list(range(300, 309)))[None, :])
+    assert np.all(res["alpha"][0] == np.float32(0.75))
+    full_check(res, K)
+
+
+def test_route_is_deterministic_and_accumulates_microbatches():
+    T, H, E, K, L = 700, 256, 768, 10, 2
+    a = route_once(T, H, E, K, L, seed=5)
+    b = route_once(T, H, E, K, L, seed=5)
+    for k in ("logits", "idx", "gate", "loads"):
+        np.testing.assert_array_equal(bits(a[k]) if a[k].dtype == np.float32 else a[k],
+                                      bits(b[k]) if b[k].dtype == np.float32 else b[k])
+    # a second call before the controller update adds to the accumulators (Algorithm 1 line 4)
+    r = a["r"]
+    r.route_step(a["x"], a["w"])
+    r.poll()
+    np.testing.assert_array_equal(np_(r.loads_peek()), 2 * a["loads"])
+
+
+# --------------------------------------------------------------- controllers
+def _drive(kind, L, E, K, steps, loads_fn, **cfg):
+    r = binding.Router(L, E, K, 64, 128, controller=kind, ki=cfg.get("ki"), kd=cfg.get("kd"), eta=cfg.get("eta"),
+                       center=cfg.get("center"))
+    center = cfg.get("center")
+    if center is None:
+        center = (kind == "id")
+    b = np.zeros((L, E), np.float32)
+    ep = np.zeros((L, E), np.float32)
+    for t in range(steps):
+        n = loads_fn(t).astype(np.int32)
+        r.loads_add(torch.from_numpy(n).cuda())
+        r.controller_update()
+        r.poll()
+        loads, bias, mxv, mnv = [np_(v) for v in r.load_stats()]
+        gates = np_(r.gate_stats())
+        _, e_prev = [np_(v) for v in r.state_export()]
+        np.testing.assert_array_equal(loads, n)
+        assert not np_(r.loads_peek()).any()               # accumulators consumed
+        for l in range(L):
+            b[l], ep[l], g, mx, mn = oracle_controller_step(
+                kind, b[l], ep[l], n[l], dict(ki=cfg.get("ki", 6e-3), kd=cfg.get("kd", 6e-3), eta=cfg.get("eta", 1e-3)),
+                center)
+            assert gates[l] == g
+            assert bits(mxv[l:l + 1])[0] == bits(np.array([mx]))[0] and bits(mnv[l:l + 1])[0] == bits(np.array([mn]))[0]
+        np.testing.assert_array_equal(bits(bias), bits(b))
+        np.testing.assert_array_equal(bits(e_prev), bits(ep))
+    return b
+
+
+def test_id_controller_closed_form_trajectories():
+    E = 768
+    half = lambda a, c: np.concatenate([np.full(384, a), np.full(384, c)])[None, :]
+    ki = kd = 2.0 ** -7
+    b = _drive("id", 1, E, 3, 20, lambda t: half(512, 1536), ki=ki, kd=kd)
+    assert np.all(b[0, :384] == np.float32(20 / 256)) and np.all(b[0, 384:] == np.float32(-20 / 256))
+    b = _drive("id", 1, E, 3, 10, lambda t: half(1024 - 16 * (t + 1), 1024 + 16 * (t + 1)), ki=ki, kd=kd)
+    assert np.all(b[0, :384] == np.float32(64 / 8192)) and np.all(b[0, 384:] == np.float32(-64 / 8192))
+
+
+@pytest.mark.parametrize("kind,E,L,center", [
+    ("id", 768, 5, None), ("id", 256, 2, 0), ("fixed_step", 768, 3, None), ("fixed_step", 768, 2, 1),
+    ("frozen", 768, 2, None), ("id", 1000, 2, None), ("id", 8, 1, None),
+])
+def test_controllers_random_loads_bit_exact(kind, E, L, center):
+    rng = np.random.default_rng(E + L)
+    K = 3
+    def loads(t):
+        hot = rng.integers(0, E, (L, 1))
+        n = rng.poisson(40, (L, E))
+        n[np.arange(L)[:, None], hot] += 500 * (t % 3)
+        n[:, 1] = 0                                   # an expert that never gets a token
+        return n
+    kw = {} if center is None else dict(center=center)
+    _drive(kind, L, E, K, 25, loads, **kw)
+
+
+def test_controller_empty_batch_reports_state_error_and_keeps_state():
+    r = binding.Router(2, 768, 10, 64, 128)
+    n = np.zeros((2, 768), np.int32)
+    n[0, :] = 7                                       # layer 0 has tokens, layer 1 has none
+    r.loads_add(torch.from_numpy(n).cuda())
+    r.controller_update()
+    assert r.poll(raise_on_error=False) == binding.MOE_ERR_STATE
+    bias, e_prev = [np_(v) for v in r.state_export()]
+    assert not bias[1].any() and not e_prev[1].any()
+    assert r.poll(raise_on_error=False) == binding.MOE_OK     # sticky status was cleared
+
+
+def test_state_export_import_resume_is_bit_identical():
+    wl = synth.WORKLOADS["tiny_top3"].with_(T=512)
+    w = synth.router_weights(wl, 0, "cuda")[None]
+    def run(steps, r):
+        for t in steps:
+            x = synth.hidden_states(wl, 0, t, "cuda")[None]
+            r.route_step(x, w)
+            r.controller_update()
+        r.poll()
+        return r
+    full = run(range(8), binding.Router(1, wl.E, wl.K, wl.H, wl.T))
+    first = run(range(4), binding.Router(1, wl.E, wl.K, wl.H, wl.T))
+    b, ep = first.state_export()
+    second = binding.Router(1, wl.E, wl.K, wl.H, wl.T)
+    second.state_import(b, ep)
+    run(range(4, 8), second)
+    for u, v in zip(full.state_export(), second.state_export()):
+        np.testing.assert_array_equal(bits(np_(u)), bits(np_(v)))
+    for u, v in zip(full.load_stats(), second.load_stats()):
+        assert torch.equal(u, v)
+
+
+# ------------------------------------------------------------- closed loops
+def _closed_loop(wl, kind, steps, check_rows=None, **kw):
+    """Teacher-forced loop: the GPU runs route + update each step; the oracle
+    replays every controller step from the GPU's loads (bitwise) and checks
+    the routing of every step against the binary32 chain."""
+    dev = "cuda"
+    r = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T, controller=kind, **kw)
+    center = (kind == "id")
+    w = torch.stack([synth.router_weights(wl, l, dev) for l in range(wl.L)])
+    b = np.zeros((wl.L, wl.E), np.float32)
+    ep = np.zeros((wl.L, wl.E), np.float32)
+    logits = torch.empty(wl.L, wl.T, wl.E, device=dev)
+    alpha = torch.empty(wl.L, wl.T, device=dev)
+    differing = checked = 0
+    hist = []
+    for t in range(steps):
+        x = torch.stack([synth.hidden_states(wl, l, t, dev) for l in range(wl.L)])
+        idx, gate = r.route_step(x, w, logits_out=logits, alpha_out=alpha)
+        r.controller_update()
+        r.poll()
+        loads, bias, mxv, mnv = [np_(v) for v in r.load_stats()]
+        lg, ix, gt, al = np_(logits), np_(idx), np_(gate), np_(alpha)
+        for l in range(wl.L):
+            oi = check_exact(lg[l], b[l], wl.K, ix[l], gt[l], al[l])
+            np.testing.assert_array_equal(loads[l], np.bincount(oi.ravel(), minlength=wl.E))
+            if check_rows is not None and t % 5 == 0:
+                d, c = check_definition(synth.bf16_bits(x[l]), synth.bf16_bits(w[l]), b[l], wl.K, lg[l], ix[l], gt[l],
+                                        rows=check_rows)
+                differing += d
+                checked += c
+            Q = oracle.quantile_target(lg[l], al[l], wl.K) if kind == "quantile" else None
+            b[l], ep[l], g, mx, mn = oracle_controller_step(
+                kind, b[l], ep[l], loads[l], dict(ki=kw.get("ki", 6e-3), kd=kw.get("kd", 6e-3), eta=kw.get("eta", 1e-3)),
+                center, Q)
+            assert bits(mxv[l:l + 1])[0] == bits(np.array([mx]))[0]
+        np.testing.assert_array_equal(bits(bias), bits(b))
+        hist.append((float(mxv.max()), float(mnv.max())))
+    if checked:
+        assert differing <= max(1, NEAR_TIE_BUDGET * checked)
+    return hist
+
+
+def test_closed_loop_tiny_top3_id():
+    # config "Tiny Top-3-of-768": 20 controller steps, fresh batch per step
+    wl = synth.WORKLOADS["tiny_top3"]
+    hist = _closed_loop(wl, "id", 20, check_rows=np.arange(0, wl.T, 4))
+    assert hist[-1][0] < hist[0][0]                    # the controller reduces the overload it started with
+
+
+@pytest.mark.parametrize("kind,K", [("id", 3), ("fixed_step", 3), ("quantile", 3), ("quantile", 5), ("id", 5)])
+def test_closed_loop_three_controllers_reduced(kind, K):
+    # the Top-3 / Top-5 single-layer comparison at a reduced token count
+    wl = synth.WORKLOADS["top3_single"].with_(T=2048, H=512, K=K)
+    hist = _closed_loop(wl, kind, 6)
+    assert all(0 <= mx <= wl.E / K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn in hist)
+
+
+def test_quantile_target_count_property_on_gpu_result():
+    # Section 2.3: with the cutoffs held fixed the new bias puts floor(mK/E)
+    # (or, with ties at the cutoff, at most that many) margins strictly above zero
+    wl = synth.WORKLOADS["top3_single"].with_(T=4096, H=256)
+    dev = "cuda"
+    r = binding.Router(1, wl.E, wl.K, wl.H, wl.T, controller="quantile")
+    x = synth.hidden_states(wl, 0, 0, dev)[None]
+    w = synth.router_weights(wl, 0, dev)[None]
+    logits = torch.empty(1, wl.T, wl.E, device=dev)
+    alpha = torch.empty(1, wl.T, device=dev)
+    r.route_step(x, w, logits_out=logits, alpha_out=alpha)
+    r.controller_update()
+    r.poll()
+    bias = np_(r.load_stats()[1])[0]
+    S = oracle.sigmoid_f32(np_(logits)[0])
+    margin = S - np_(alpha)[0][:, None]
+    q = (wl.T * wl.K) // wl.E
+    above = (margin > -bias[None, :]).sum(0)
+    at_or_above = (margin >= -bias[None, :]).sum(0)
+    assert np.all(above <= q) and np.all(at_or_above >= q + 1)
+    with pytest.raises(binding.MoeRouteError):          # needs a fresh dump per update
+        r.controller_update()
+
+
+def test_host_buffer_step_matches_device_step():
+    T, H, E, K, L = 900, 256, 768, 10, 2
+    res = route_once(T, H, E, K, L, seed=9)
+    r = binding.Router(L, E, K, H, T, host_staging=True)
+    xh, wh = res["x"].cpu().pin_memory(), res["w"].cpu().pin_memory()
+    ih = torch.empty(L, T, K, dtype=torch.int32).pin_memory()
+    gh = torch.empty(L, T, K, dtype=torch.float32).pin_memory()
+    r.route_step_host(xh, wh, ih, gh)
+    r.poll()
+    np.testing.assert_array_equal(ih.numpy(), res["idx"])
+    np.testing.assert_array_equal(bits(gh.numpy()), bits(res["gate"]))
+    np.testing.assert_array_equal(np_(r.loads_peek()), res["loads"])
+
+
+def test_argument_errors_are_reported_not_raised_by_cuda():
+    r = binding.Router(1, 768, 10, 64, 128)
+    x = torch.zeros(1, 256, 64, device="cuda", dtype=torch.bfloat16)
+    w = torch.zeros(1, 768, 64, device="cuda", dtype=torch.bfloat16)
+    with pytest.raises(binding.MoeRouteError) as ei:
+        r.route_step(x, w)                               # more tokens than max_tokens
+    assert ei.value.code == binding.MOE_ERR_INVALID_ARG
+    rq = binding.Router(1, 768, 3, 64, 128, controller="quantile")
+    with pytest.raises(binding.MoeRouteError):
+        rq.route_step(x[:, :128].contiguous(), w)        # quantile controller without the dump buffers
+    with pytest.raises(binding.MoeRouteError):
+        binding.Router(2, 768, 3, 64, 128, controller="quantile")
+    assert r.poll(raise_on_error=False) == binding.MOE_OK
+
+
+# ------------------------------------------------ full-size configurations
+def _full_size(wl, layers, steps=1, sample=192):
+    """Full T and H of a configuration (a few layers of it), in the launch
+    configuration the benchmark times.  All tokens against the binary32
+    chain; a seeded token sample against the fp64 definition."""
+    dev = "cuda"
+    wl = wl.with_(L=layers)
+    r = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T)
+    w = torch.stack([synth.router_weights(wl, l, dev) for l in range(wl.L)])
+    b = np.zeros((wl.L, wl.E), np.float32)
+    rng = np.random.default_rng(wl.wid)
+    differing = checked = 0
+    for t in range(steps):
+        x = torch.stack([synth.hidden_states(wl, l, t, dev) for l in range(wl.L)])
+        idx, gate = r.route_step(x, w)                  # the timed configuration: no dump
+        r.poll()
+        loads = np_(r.loads_peek())
+        ix, gt = np_(idx), np_(gate)
+        assert loads.sum() == wl.L * wl.T * wl.K
+        for l in range(wl.L):
+            np.testing.assert_array_equal(loads[l], np.bincount(ix[l].ravel(), minlength=wl.E))
+        # same inputs once more with the dump, one layer at a time, for the element-wise checks
+        r2 = binding.Router(1, wl.E, wl.K, wl.H, wl.T)
+        for l in range(wl.L):
+            r2.state_import(bias=torch.from_numpy(b[l:l + 1]).cuda())
+            logits = torch.empty(1, wl.T, wl.E, device=dev)
+            i2, g2 = r2.route_step(x[l:l + 1].contiguous(), w[l:l + 1].contiguous(), logits_out=logits)
+            r2.poll()
+            np.testing.assert_array_equal(np_(i2)[0], ix[l])        # dump on/off changes nothing
+            np.testing.assert_array_equal(bits(np_(g2)[0]), bits(gt[l]))
+            lg = np_(logits)[0]
+            check_exact(lg, b[l], wl.K, ix[l], gt[l])
+            rows = np.sort(rng.choice(wl.T, sample, replace=False))
+            d, c = check_definition(synth.bf16_bits(x[l]), synth.bf16_bits(w[l]), b[l], wl.K, lg, ix[l], gt[l], rows)
+            differing += d
+            checked += c
+        r.controller_update()
+        r.poll()
+        b = np_(r.load_stats()[1])
+    assert differing <= max(1, NEAR_TIE_BUDGET * checked)
+
+
+def test_full_size_top10_single_layer():
+    _full_size(synth.WORKLOADS["top10_single"], layers=1, steps=2)
+
+
+def test_full_size_top3_and_top5_single_layer():
+    _full_size(synth.WORKLOADS["top3_single"], layers=1)
+    _full_size(synth.WORKLOADS["top5_single"], layers=1)
+
+
+def test_full_size_deep_stack_layers():
+    _full_size(synth.WORKLOADS["top10_deep"], layers=3, steps=2, sample=96)
+
+
+def test_full_size_large_scale_layers():
+    _full_size(synth.WORKLOADS["top10_large"], layers=2, sample=64)
