@@ -149,6 +149,13 @@ int moe_state_import(moe_route_ctx* ctx, const float* bias, const float* e_prev,
  * status (MOE_OK, MOE_ERR_TIMEOUT, MOE_ERR_STATE, MOE_ERR_CUDA); clears it. */
 int moe_route_poll(moe_route_ctx* ctx);
 
+/* Validation utility for the candidate filter of moe_route_step: sweeps every
+ * finite fp32 logit and writes to dev_result[0] (device, one float) the largest
+ * absolute difference between the approximate score used for filtering and the
+ * exact score of Section 2.2.  The filter is sound while this stays below the
+ * slack compiled into the kernel (2e-6). */
+int moe_debug_score_gap(float* dev_result, void* cuda_stream);
+
 /* Number of kernels this context has launched so far. */
 int64_t moe_route_launch_count(const moe_route_ctx* ctx);
 

@@ -23,7 +23,7 @@ CONTROLLERS = {"id": MOE_CTRL_ID, "fixed_step": MOE_CTRL_FIXED_STEP, "quantile":
 SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_init", "moe_route_step",
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
-           "moe_last_error", "moe_route_destroy"]
+           "moe_last_error", "moe_route_destroy", "moe_debug_score_gap"]
 
 
 class MoeRouteConfig(C.Structure):
@@ -72,6 +72,7 @@ def load():
     L.moe_last_error.argtypes = [vp]
     L.moe_last_error.restype = C.c_char_p
     L.moe_route_destroy.argtypes = [vp]
+    L.moe_debug_score_gap.argtypes = [vp, vp]
     _lib = L
     return L
 
@@ -88,6 +89,15 @@ def _ptr(t):
 
 def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def debug_score_gap(device="cuda") -> float:
+    """Largest |approximate score - exact score| over all finite fp32 logits (runs on the GPU)."""
+    out = torch.zeros(1, dtype=torch.float32, device=device)
+    rc = load().moe_debug_score_gap(_ptr(out), _stream())
+    if rc != MOE_OK:
+        raise MoeRouteError(rc, "moe_debug_score_gap failed")
+    return float(out.item())
 
 
 class Router:

@@ -147,11 +147,11 @@ int launch_route(moe_route_ctx* ctx, const RouteParams& rp, int grid, cudaStream
   static bool attr_set[64] = {};
   const size_t smem = route_smem_bytes<KL>();
   if (!attr_set[ctx->device & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(route_step_kernel<KL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(route_step_kernel<KL, (KL <= 16)>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(route_step_kernel)");
     attr_set[ctx->device & 63] = true;
   }
-  route_step_kernel<KL><<<grid, kRouteThreads, smem, st>>>(ctx->tm_x, ctx->tm_w, rp);
+  route_step_kernel<KL, (KL <= 16)><<<grid, kRouteThreads, smem, st>>>(ctx->tm_x, ctx->tm_w, rp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "route_step_kernel launch");
   ctx->launches += 1;
@@ -437,6 +437,29 @@ int moe_route_poll(moe_route_ctx* ctx) {
     return fail(ctx, st[0], "device status %d", st[0]);
   }
   return MOE_OK;
+}
+
+// grid-stride sweep over all 2^32 fp32 bit patterns (NaN and infinities skipped)
+__global__ void score_gap_kernel(unsigned int* out) {
+  float worst = 0.0f;
+  const unsigned long long n = 1ull << 32;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned int bits = (unsigned int)i;
+    if ((bits & 0x7f800000u) == 0x7f800000u) continue;
+    const float z = __uint_as_float(bits);
+    worst = fmaxf(worst, fabsf(moe::approx_score(z) - moe::sigmoid_score(z)));
+  }
+  for (int d = 16; d > 0; d >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, d));
+  if ((threadIdx.x & 31) == 0) atomicMax(out, __float_as_uint(worst));
+}
+
+int moe_debug_score_gap(float* dev_result, void* cuda_stream) {
+  if (!dev_result) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(dev_result, 0, sizeof(float), st) != cudaSuccess) return MOE_ERR_CUDA;
+  score_gap_kernel<<<148 * 8, 256, 0, st>>>(reinterpret_cast<unsigned int*>(dev_result));
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 int64_t moe_route_launch_count(const moe_route_ctx* ctx) { return ctx ? ctx->launches : 0; }

@@ -93,6 +93,13 @@ def test_route_is_deterministic_and_accumulates_microbatches():
     np.testing.assert_array_equal(np_(r.loads_peek()), 2 * a["loads"])
 
 
+def test_candidate_filter_slack_covers_every_fp32_logit():
+    # the approximate score only pre-selects candidates; it must stay within the
+    # compiled slack (absolute part 4e-6, of which half is the budget) of the exact score
+    gap = binding.debug_score_gap()
+    assert 0.0 < gap < 2e-6, gap
+
+
 # --------------------------------------------------------------- controllers
 def _drive(kind, L, E, K, steps, loads_fn, **cfg):
     r = binding.Router(L, E, K, 64, 128, controller=kind, ki=cfg.get("ki"), kd=cfg.get("kd"), eta=cfg.get("eta"),
