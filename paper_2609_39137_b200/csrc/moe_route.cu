@@ -145,13 +145,13 @@ int encode_map(moe_route_ctx* ctx, CUtensorMap* out, const void* base, uint64_t 
 template <int KL>
 int launch_route(moe_route_ctx* ctx, const RouteParams& rp, int grid, cudaStream_t st) {
   static bool attr_set[64] = {};
-  const size_t smem = route_smem_bytes<KL>();
+  const size_t smem = route_smem_bytes();
   if (!attr_set[ctx->device & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(route_step_kernel<KL, (KL <= 16)>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(route_step_kernel<KL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(route_step_kernel)");
     attr_set[ctx->device & 63] = true;
   }
-  route_step_kernel<KL, (KL <= 16)><<<grid, kRouteThreads, smem, st>>>(ctx->tm_x, ctx->tm_w, rp);
+  route_step_kernel<KL><<<grid, kRouteThreads, smem, st>>>(ctx->tm_x, ctx->tm_w, rp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "route_step_kernel launch");
   ctx->launches += 1;
@@ -461,6 +461,20 @@ int moe_debug_score_gap(float* dev_result, void* cuda_stream) {
   score_gap_kernel<<<148 * 8, 256, 0, st>>>(reinterpret_cast<unsigned int*>(dev_result));
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
+
+#ifdef MOE_KERNEL_TIMERS
+// debug builds only: cycle accounting of the route kernel, 32 counters, optionally reset
+int moe_debug_read_timers(long long* host_out, int reset) {
+  cudaDeviceSynchronize();
+  if (host_out && cudaMemcpyFromSymbol(host_out, moe::g_route_timers, sizeof(long long) * 32) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (reset) {
+    long long z[32] = {0};
+    if (cudaMemcpyToSymbol(moe::g_route_timers, z, sizeof z) != cudaSuccess) return MOE_ERR_CUDA;
+  }
+  return MOE_OK;
+}
+#endif
 
 int64_t moe_route_launch_count(const moe_route_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
