@@ -166,14 +166,14 @@ int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, in
       return fail(ctx, MOE_ERR_INVALID_ARG, "x and w must be 16-byte aligned");
     int rc = encode_map(ctx, &ctx->tm_x, x, c.hidden, T, c.num_layers, kBM);
     if (rc) return rc;
-    rc = encode_map(ctx, &ctx->tm_w, w, c.hidden, c.num_experts, c.num_layers, kBN);
+    rc = encode_map(ctx, &ctx->tm_w, w, c.hidden, c.num_experts, c.num_layers, kBN / 2);
     if (rc) return rc;
     ctx->map_x_ptr = x; ctx->map_w_ptr = w; ctx->map_tokens = T;
   }
   RouteParams rp{};
   rp.L = c.num_layers; rp.T = T; rp.H = c.hidden; rp.E = c.num_experts; rp.K = c.top_k;
-  rp.tiles_per_layer = (T + kBM - 1) / kBM;
-  rp.num_items = rp.tiles_per_layer * c.num_layers;
+  rp.pairs_per_layer = (T + 2 * kBM - 1) / (2 * kBM);
+  rp.num_items = rp.pairs_per_layer * c.num_layers;
   rp.num_kblocks = (c.hidden + kBK - 1) / kBK;
   rp.num_chunks = (c.num_experts + kBN - 1) / kBN;
   rp.bias = at<float>(ctx, ctx->lay.bias);
@@ -181,7 +181,8 @@ int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, in
   rp.topk_idx = idx; rp.topk_gate = gate; rp.logits_out = logits; rp.alpha_out = alpha;
   rp.status = status_ptr(ctx);
   rp.spin_limit = c.spin_limit > 0 ? (uint32_t)c.spin_limit : 0x7fffffffu;
-  const int grid = rp.num_items < ctx->num_sms ? rp.num_items : ctx->num_sms;
+  const int max_pairs = ctx->num_sms / 2;
+  const int grid = 2 * (rp.num_items < max_pairs ? rp.num_items : max_pairs);   // clusters of 2 CTAs
   const int need = c.top_k + (alpha ? 1 : 0);
   if (need <= 3) return launch_route<3>(ctx, rp, grid, st);
   if (need <= 5) return launch_route<5>(ctx, rp, grid, st);
@@ -470,6 +471,7 @@ int moe_debug_read_timers(long long* host_out, int reset) {
     return MOE_ERR_CUDA;
   if (reset) {
     long long z[32] = {0};
+    z[24] = 0x7fffffffffffffffll;   // running minimum of the CTA start times
     if (cudaMemcpyToSymbol(moe::g_route_timers, z, sizeof z) != cudaSuccess) return MOE_ERR_CUDA;
   }
   return MOE_OK;
