@@ -156,6 +156,37 @@ int moe_route_poll(moe_route_ctx* ctx);
  * slack compiled into the kernel (2e-6). */
 int moe_debug_score_gap(float* dev_result, void* cuda_stream);
 
+/* Quantile target without any allocation and without a context (the paper has
+ * no counterpart for this call; it computes the same Q_j as the quantile
+ * controller's update does from its dump).
+ *
+ * Meant for callers that cannot obtain device memory when they need this
+ * result and have no workspace of their own to lend: for instance a serving
+ * process that handed all of its device memory to its own pool at start-up, or
+ * a latency-critical loop in which the implicit synchronisation and the
+ * possible failure of cudaMalloc are not acceptable.  The radix-select scratch
+ * (a histogram of 256 bins per expert plus two words per expert) therefore
+ * lives in a fixed array inside the library: 1,056,768 bytes, present on every
+ * device that loads the library until the process exits.  That caps the call at
+ * num_experts <= 1024; more returns MOE_ERR_WORKSPACE and launches nothing.
+ * num_tokens is not limited.
+ *
+ *   logits     [num_tokens][num_experts] float32, device (a dump of moe_route_step)
+ *   alpha      [num_tokens] float32, device ((K+1)-th largest biased score per token)
+ *   target_out [num_experts] float32, device: Q_j = -(r-th smallest of
+ *              sigmoid(logits[i][j]) - alpha[i] over i), r = m - floor(m K / E)
+ *
+ * The first call on a device looks up the device address of the array and the
+ * SM count (nothing is allocated); make that first call with the device current
+ * and before any stream capture starts.  Later calls only launch kernels.
+ * All calls share the one array and it keeps what the previous call left, so
+ * every call first clears what must start at zero -- and two calls whose kernels
+ * can overlap on the GPU (different streams, no ordering between them) race on
+ * it.  Asynchronous on the stream; returns MOE_OK, MOE_ERR_INVALID_ARG,
+ * MOE_ERR_WORKSPACE, MOE_ERR_UNSUPPORTED (device ordinal >= 64) or MOE_ERR_CUDA. */
+int moe_quantile_target_static(const float* logits, const float* alpha, int32_t num_tokens,
+                               int32_t num_experts, int32_t top_k, float* target_out, void* cuda_stream);
+
 /* Number of kernels this context has launched so far. */
 int64_t moe_route_launch_count(const moe_route_ctx* ctx);
 

@@ -23,7 +23,7 @@ CONTROLLERS = {"id": MOE_CTRL_ID, "fixed_step": MOE_CTRL_FIXED_STEP, "quantile":
 SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_init", "moe_route_step",
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
-           "moe_last_error", "moe_route_destroy", "moe_debug_score_gap"]
+           "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static"]
 
 
 class MoeRouteConfig(C.Structure):
@@ -73,6 +73,7 @@ def load():
     L.moe_last_error.restype = C.c_char_p
     L.moe_route_destroy.argtypes = [vp]
     L.moe_debug_score_gap.argtypes = [vp, vp]
+    L.moe_quantile_target_static.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     _lib = L
     return L
 
@@ -98,6 +99,20 @@ def debug_score_gap(device="cuda") -> float:
     if rc != MOE_OK:
         raise MoeRouteError(rc, "moe_debug_score_gap failed")
     return float(out.item())
+
+
+def quantile_target_static(logits, alpha, top_k, target_out):
+    """moe_quantile_target_static: Q_j for one layer from a logits dump, using only the scratch array built
+    into the library (no allocation happens in the call; `target_out` is the caller's [E] float32 tensor).
+    Calls that may overlap on the GPU must not be issued concurrently: they share the one scratch array."""
+    m, E = logits.shape
+    assert logits.dtype == torch.float32 and alpha.dtype == torch.float32 and target_out.dtype == torch.float32
+    assert logits.is_contiguous() and alpha.numel() == m and target_out.numel() == E
+    rc = load().moe_quantile_target_static(_ptr(logits), _ptr(alpha), m, E, top_k, _ptr(target_out), _stream())
+    if rc != MOE_OK:
+        raise MoeRouteError(rc, "moe_quantile_target_static failed"
+                            + (": more experts than the built-in scratch holds (1024)" if rc == MOE_ERR_WORKSPACE else ""))
+    return target_out
 
 
 class Router:

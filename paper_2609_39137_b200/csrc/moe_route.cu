@@ -9,6 +9,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "controller_kernel.cuh"
@@ -82,6 +83,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 }  // namespace
+
+// Scratch of moe_quantile_target_static: radix histogram [1024][256] u32, then prefix [1024] and
+// rank [1024] u32.  Lives in every device that loads the library, until the process exits.
+constexpr int kStaticMaxExperts = 1024;
+constexpr int kStaticMaxDevices = 64;
+constexpr size_t kStaticScratchBytes = (size_t)kStaticMaxExperts * 256 * 4 + 2 * (size_t)kStaticMaxExperts * 4;
+static __device__ __align__(256) unsigned char moe_static_quantile_scratch[kStaticScratchBytes];
+static void* g_static_scratch_dev[kStaticMaxDevices];   // device address of the array, per device
+static int g_static_sms[kStaticMaxDevices];
+static std::mutex g_static_mu;
 
 struct moe_route_ctx {
   moe_route_config cfg;
@@ -477,6 +488,52 @@ int moe_debug_read_timers(long long* host_out, int reset) {
   return MOE_OK;
 }
 #endif
+
+int moe_quantile_target_static(const float* logits, const float* alpha, int32_t num_tokens, int32_t num_experts,
+                               int32_t top_k, float* target_out, void* cuda_stream) {
+  if (!logits || !alpha || !target_out) return MOE_ERR_INVALID_ARG;
+  if (num_tokens < 1 || num_experts < 1 || top_k < 1 || top_k >= num_experts) return MOE_ERR_INVALID_ARG;
+  if (num_experts > kStaticMaxExperts) return MOE_ERR_WORKSPACE;   // beyond the built-in scratch
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+  if (dev < 0 || dev >= kStaticMaxDevices) return MOE_ERR_UNSUPPORTED;
+  {
+    // once per device, with that device current: turn the host-side stand-in of the array into its
+    // device address (the symbol itself is not a device pointer and must never reach a kernel argument)
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (g_static_scratch_dev[dev] == nullptr) {
+      void* ptr = nullptr;
+      cudaError_t e = cudaGetSymbolAddress(&ptr, moe_static_quantile_scratch);
+      if (e != cudaSuccess || ptr == nullptr) return MOE_ERR_CUDA;
+      int sms = 0;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return MOE_ERR_CUDA;
+      g_static_sms[dev] = sms;
+      g_static_scratch_dev[dev] = ptr;
+    }
+  }
+  uint8_t* base = static_cast<uint8_t*>(g_static_scratch_dev[dev]);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  QbParams q{};
+  q.logits = logits; q.alpha = alpha; q.m = num_tokens; q.E = num_experts; q.K = top_k;
+  q.hist = reinterpret_cast<uint32_t*>(base);
+  q.prefix = reinterpret_cast<uint32_t*>(base + (size_t)kStaticMaxExperts * 256 * 4);
+  q.rank = q.prefix + kStaticMaxExperts;
+  q.target = target_out;
+  // the array keeps whatever the previous call left: the init kernel clears the histogram and
+  // resets prefix and rank before anything is counted
+  qb_init_kernel<<<64, 256, 0, st>>>(q);
+  const int col_groups = (num_experts + kQbCols - 1) / kQbCols;
+  int splits = (2 * g_static_sms[dev] + col_groups - 1) / col_groups;
+  const int max_splits = (num_tokens + 63) / 64;
+  if (splits > max_splits) splits = max_splits;
+  if (splits < 1) splits = 1;
+  for (int pass = 0; pass < 4; ++pass) {
+    qb_hist_kernel<<<dim3(col_groups, splits), kQbThreads, 0, st>>>(q, pass);
+    qb_scan_kernel<<<(num_experts * 32 + 255) / 256, 256, 0, st>>>(q, pass);
+  }
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
 
 int64_t moe_route_launch_count(const moe_route_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
