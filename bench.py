@@ -36,7 +36,7 @@ RING = 8   # distinct input batches cycled through, so every timed step reads x 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one route_step_kernel launch, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the workload)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"top10_single": 70723840 + 2969600}   # profiles/route_step_kernel_top10_single.md
 
 
 def peaks():
