@@ -42,6 +42,9 @@ __global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlPara
   __shared__ long long total_s;
   __shared__ int max_s, min_s;
 
+  // launched with programmatic stream serialisation: the block may already be resident while the
+  // routing kernel before it drains; nothing of that kernel's output is touched before this returns
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int layer = blockIdx.x;
   const int i = threadIdx.x;
   const int lane = i & 31, warp = i >> 5;

@@ -355,7 +355,21 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
   p.gate_count = at<int>(ctx, ctx->lay.gate_count);
   p.qb_target = at<float>(ctx, ctx->lay.qb_target);
   p.status = status_ptr(ctx);
-  controller_kernel<<<c.num_layers, kCtrlThreads, 0, st>>>(p);
+  {
+    // programmatic stream serialisation: the launch latency overlaps the tail of the kernel before it
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(c.num_layers);
+    lc.blockDim = dim3(kCtrlThreads);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &attr;
+    lc.numAttrs = 1;
+    cudaError_t le = cudaLaunchKernelEx(&lc, controller_kernel, p);
+    if (le != cudaSuccess) return cuda_fail(ctx, le, "controller_kernel launch");
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "controller_kernel launch");
   ctx->launches += 1;
