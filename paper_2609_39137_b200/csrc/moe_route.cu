@@ -186,6 +186,10 @@ int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, in
   rp.pairs_per_layer = (T + 2 * kBM - 1) / (2 * kBM);
   rp.num_items = rp.pairs_per_layer * c.num_layers;
   rp.num_kblocks = (c.hidden + kBK - 1) / kBK;
+  // fp32 accumulation error of the tensor core grows with the length of the accumulation chain: chains
+  // longer than 2048 hidden elements are split in two and added once in fp32 by the epilogue
+  rp.num_segs = (c.hidden > 2048) ? 2 : 1;
+  rp.seg_kblocks = (rp.num_kblocks + rp.num_segs - 1) / rp.num_segs;
   rp.num_chunks = (c.num_experts + kBN - 1) / kBN;
   rp.bias = at<float>(ctx, ctx->lay.bias);
   rp.loads = at<int>(ctx, ctx->lay.loads_acc);
