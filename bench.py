@@ -34,9 +34,9 @@ METRIC = "routed_tokens_per_s"
 UNIT = "tokens/s"
 RING = 8   # distinct input batches cycled through, so every timed step reads x from HBM
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one route_step_kernel launch, from the ncu
-# capture summarised under profiles/ (None until a capture exists for the workload)
-NCU_TRAFFIC_BYTES = {"top10_single": 70723840 + 2969600}   # profiles/route_step_kernel_top10_single.md
+# dram__bytes_read.sum + dram__bytes_write.sum of one route_step_kernel launch, from an ncu capture of
+# this command on the same workload (the summary is kept with the other profile summaries); None = no capture
+NCU_TRAFFIC_BYTES = {"top10_single": 70723840 + 2969600}
 
 
 def peaks():
