@@ -65,6 +65,9 @@ def lib():
             L.oracle_quantile_target.argtypes = [_f32p, _f32p, _i64, _i64, _i64, _f32p]
             L.oracle_quantile_update.argtypes = [_f32p, _f32p, _f32p, _f32p, _i64, C.c_float, C.c_int]
             L.oracle_violations.argtypes = [_i64p, _i64, _f32p, _f32p]
+            L.oracle_load_diagnostics.argtypes = [_i64p, _i32p, _f32p, _f32p, _i64, _f32p]
+            L.oracle_gate_entropy_mean.argtypes = [_f32p, _i64, _i64]
+            L.oracle_gate_entropy_mean.restype = C.c_double
             L.oracle_route_tokens_f64.argtypes = [_u16p, _u16p, _f32p, _i64, _i64, _i64, _i64,
                                                   _f64p, _i32p, _f64p, _f64p, _f64p, _i64p]
             _lib = L
@@ -258,3 +261,23 @@ def violations(n):
     if lib().oracle_violations(_p(n, _i64p), n.shape[0], C.byref(mx), C.byref(mn)):
         raise ValueError("empty batch: sum of loads is zero")
     return np.float32(mx.value), np.float32(mn.value)
+
+
+def load_diagnostics(n, gate, b_old, b_new):
+    """(gate fraction, busiest-10 % share, inactive-expert ratio, mean |delta b|) as binary32 values."""
+    n = _arr(n, np.int64)
+    gate = _arr(gate, np.int32)
+    b_old = _arr(b_old, np.float32)
+    b_new = _arr(b_new, np.float32)
+    out = np.empty(4, np.float32)
+    if lib().oracle_load_diagnostics(_p(n, _i64p), _p(gate, _i32p), _p(b_old, _f32p), _p(b_new, _f32p),
+                                     n.shape[0], _p(out, _f32p)):
+        raise ValueError("empty batch: sum of loads is zero")
+    return out
+
+
+def gate_entropy_mean(gate):
+    """Mean over tokens of H = -sum_k w_k ln w_k (nats), Section 4.3."""
+    gate = _arr(gate, np.float32)
+    T, K = gate.shape
+    return float(lib().oracle_gate_entropy_mean(_p(gate, _f32p), T, K))

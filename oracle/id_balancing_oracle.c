@@ -383,6 +383,69 @@ int oracle_violations(const int64_t *n, int64_t E, float *maxvio,
 }
 
 /*
+ * Load-control diagnostics the paper plots (Section 3 figure captions, Section 4.3), per layer:
+ *   gate_frac     fraction of experts whose worsening gate g_i is open (Eq. 11)
+ *   busiest_share share of all token assignments that went to the busiest 10 % of
+ *                 the experts (balanced value 0.10).  Reading: "10 % of the experts"
+ *                 is m = E/10 rounded to the nearest integer (at least 1).
+ *   inactive      fraction of experts that received no token
+ *   bias_drift    mean absolute bias change (1/E) sum |b_new - b_old|
+ * All in binary64, rounded once to binary32.  out[4] in the order above.
+ */
+static int cmp_i64_desc(const void *pa, const void *pb)
+{
+    int64_t a = *(const int64_t *)pa, b = *(const int64_t *)pb;
+    return (a < b) - (a > b);
+}
+
+int oracle_load_diagnostics(const int64_t *n, const int32_t *gate, const float *b_old,
+                            const float *b_new, int64_t E, float *out)
+{
+    int64_t *sorted = (int64_t *)malloc((size_t)E * sizeof *sorted);
+    if (!sorted) return -1;
+    int64_t total = 0, open_gates = 0, empty = 0;
+    double drift = 0.0;
+    for (int64_t i = 0; i < E; ++i) {
+        sorted[i] = n[i];
+        total += n[i];
+        open_gates += gate[i] ? 1 : 0;
+        empty += (n[i] == 0);
+        drift += fabs((double)b_new[i] - (double)b_old[i]);
+    }
+    if (total <= 0) { free(sorted); return -1; }
+    qsort(sorted, (size_t)E, sizeof *sorted, cmp_i64_desc);
+    int64_t m = (E + 5) / 10;
+    if (m < 1) m = 1;
+    int64_t top = 0;
+    for (int64_t i = 0; i < m; ++i) top += sorted[i];
+    out[0] = (float)((double)open_gates / (double)E);
+    out[1] = (float)((double)top / (double)total);
+    out[2] = (float)((double)empty / (double)E);
+    out[3] = (float)(drift / (double)E);
+    free(sorted);
+    return 0;
+}
+
+/*
+ * Top-K gating-score entropy (Section 4.3): H = - sum_{k<K} w_k ln w_k in nats,
+ * w the normalised combination weights of a token; returns the mean over the
+ * T tokens (0 ln 0 = 0).  gate : [T][K] binary32.
+ */
+double oracle_gate_entropy_mean(const float *gate, int64_t T, int64_t K)
+{
+    double sum = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+        double h = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            double w = (double)gate[t * K + k];
+            if (w > 0.0) h -= w * log(w);
+        }
+        sum += h;
+    }
+    return sum / (double)T;
+}
+
+/*
  * One whole routing pass of the definition for a slice of tokens: logits,
  * scores, biased top-K, gates and load counts (Section 2.2, Algorithm 1
  * lines 3-4).  Convenience for timing and for tests; it only chains the

@@ -50,6 +50,8 @@ WORKLOADS = {
     "top5_single": Workload("top5_single", 1, 16384, 2048, 768, 5, 16, 1.0, 0.05, 200, wid=3),
     "top10_deep": Workload("top10_deep", 48, 16384, 2048, 768, 10, 16, 1.0, 0.05, 500, drift=True, wid=4),
     "top10_large": Workload("top10_large", 60, 65536, 4096, 768, 10, 32, 1.0, 0.05, 100, wid=5),
+    # the paper's second routing shape (Table A, medium model): Top-8 of 256 experts, hidden 2048, 28 layers
+    "top8_of_256": Workload("top8_of_256", 28, 16384, 2048, 256, 8, 16, 1.0, 0.05, 100, wid=6),
 }
 
 

@@ -438,6 +438,47 @@ def test_violation_bounds(row):
     assert mx == 0 and mn == 0
 
 
+# ------------------------------------------------------------- diagnostics
+def test_load_diagnostics_closed_forms():
+    E = 768
+    # perfectly balanced: busiest 10 % of the experts (77 of 768) hold 77/768 of the assignments (target 0.10)
+    n = np.full(E, 40, np.int64)
+    z = np.zeros(E, np.float32)
+    g = np.zeros(E, np.int32)
+    d = oracle.load_diagnostics(n, g, z, z)
+    assert abs(d[1] - 77 / 768) < 1e-7 and d[0] == 0 and d[2] == 0 and d[3] == 0
+    # everything on 3 experts: share 1, inactive ratio (E-3)/E
+    n = np.zeros(E, np.int64)
+    n[[5, 100, 700]] = [10, 20, 30]
+    g[:192] = 1
+    b0 = np.zeros(E, np.float32)
+    b1 = np.full(E, 0.25, np.float32)
+    b1[::2] = -0.25
+    d = oracle.load_diagnostics(n, g, b0, b1)
+    assert d[1] == 1.0 and abs(d[2] - 765 / 768) < 1e-7 and d[0] == np.float32(0.25) and d[3] == np.float32(0.25)
+    # share against an explicit partial sort
+    rng = np.random.default_rng(70)
+    n = rng.integers(0, 500, E).astype(np.int64)
+    d = oracle.load_diagnostics(n, g, b0, b0)
+    np.testing.assert_allclose(d[1], np.sort(n)[::-1][:77].sum() / n.sum(), rtol=1e-7)
+    assert oracle.load_diagnostics(np.arange(1, 11, dtype=np.int64), np.zeros(10, np.int32), z[:10], z[:10])[1] == np.float32(10 / 55)
+
+
+def test_gate_entropy_closed_forms():
+    # uniform weights over K experts: H = ln K; a one-hot weight vector: H = 0
+    for K in (3, 8, 10):
+        w = np.full((7, K), 1.0 / K, np.float32)
+        assert abs(oracle.gate_entropy_mean(w) - np.log(K)) < 1e-6
+    w = np.zeros((4, 5), np.float32)
+    w[:, 2] = 1.0
+    assert oracle.gate_entropy_mean(w) == 0.0
+    rng = np.random.default_rng(71)
+    w = rng.random((50, 10)).astype(np.float32)
+    w /= w.sum(1, keepdims=True)
+    ref = scipy.special.entr(w.astype(np.float64)).sum(1).mean()
+    assert abs(oracle.gate_entropy_mean(w) - ref) < 1e-12
+
+
 # ------------------------------------------------------------- whole chain
 def test_route_tokens_chain_and_threads_agree():
     from paper_2609_39137_b200 import synth
