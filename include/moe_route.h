@@ -135,6 +135,20 @@ int moe_load_stats(moe_route_ctx* ctx, int32_t* loads, float* bias, float* maxvi
  * recent ID update: gate_count [L] int32. */
 int moe_gate_stats(moe_route_ctx* ctx, int32_t* gate_count, void* cuda_stream);
 
+/* Diagnostics of the most recent controller update, as plotted in the paper
+ * (figure captions of Section 3; Section 4.3): diag [L][4] float32 (device) =
+ * { fraction of open worsening gates (Eq. 11), share of all token assignments
+ * that went to the busiest 10 % of the experts (round(E/10) experts; 0.10 when
+ * balanced), fraction of experts that received no token, mean |bias change| of
+ * the update }. */
+int moe_load_diagnostics(moe_route_ctx* ctx, float* diag, void* cuda_stream);
+
+/* Mean over the tokens of a routing step of the top-K gating-score entropy
+ * H = -sum_k w_k ln w_k (nats, Section 4.3), per layer: topk_gate
+ * [L][num_tokens][K] as written by moe_route_step, entropy [L] float32 (device). */
+int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tokens, float* entropy,
+                     void* cuda_stream);
+
 /* Load accumulators not yet consumed: read them, or add external counts
  * (Algorithm 1 line 4: counts are summed over microbatches and the
  * data-parallel group -- a caller that shards tokens adds its peers' counts). */

@@ -23,7 +23,8 @@ CONTROLLERS = {"id": MOE_CTRL_ID, "fixed_step": MOE_CTRL_FIXED_STEP, "quantile":
 SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_init", "moe_route_step",
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
-           "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static"]
+           "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static",
+           "moe_load_diagnostics", "moe_gate_entropy"]
 
 
 class MoeRouteConfig(C.Structure):
@@ -62,6 +63,8 @@ def load():
     L.moe_controller_update.argtypes = [vp, vp]
     L.moe_load_stats.argtypes = [vp, vp, vp, vp, vp, vp]
     L.moe_gate_stats.argtypes = [vp, vp, vp]
+    L.moe_load_diagnostics.argtypes = [vp, vp, vp]
+    L.moe_gate_entropy.argtypes = [vp, vp, i32, vp, vp]
     L.moe_loads_peek.argtypes = [vp, vp, vp]
     L.moe_loads_add.argtypes = [vp, vp, vp]
     L.moe_state_export.argtypes = [vp, vp, vp, vp]
@@ -186,6 +189,20 @@ class Router:
         g = torch.empty(self.L, dtype=torch.int32, device=self.device)
         self._check(self.lib.moe_gate_stats(self.h, _ptr(g), _stream()))
         return g
+
+    def load_diagnostics(self):
+        """[L][4]: open-gate fraction, busiest-10 % share, inactive-expert ratio, mean |bias change|."""
+        d = torch.empty(self.L, 4, dtype=torch.float32, device=self.device)
+        self._check(self.lib.moe_load_diagnostics(self.h, _ptr(d), _stream()))
+        return d
+
+    def gate_entropy(self, topk_gate):
+        """[L]: mean top-K gate entropy (nats) of the given routing step's gates [L][T][K]."""
+        T = topk_gate.shape[-2]
+        assert topk_gate.dtype == torch.float32 and topk_gate.is_contiguous() and topk_gate.numel() == self.L * T * self.K
+        h = torch.empty(self.L, dtype=torch.float32, device=self.device)
+        self._check(self.lib.moe_gate_entropy(self.h, _ptr(topk_gate), T, _ptr(h), _stream()))
+        return h
 
     def loads_peek(self):
         loads = torch.empty(self.L, self.E, dtype=torch.int32, device=self.device)

@@ -26,6 +26,7 @@ struct CtrlParams {
   int center;
   float* bias;        // [L][E] in/out
   float* e_prev;      // [L][E] in/out
+  float* bias_prev;   // [L][E] out: bias before this update (for the drift diagnostic)
   int* loads_acc;     // [L][E] consumed and zeroed
   int* loads_last;    // [L][E] out
   float* maxvio;      // [L] out
@@ -127,6 +128,7 @@ __global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlPara
   __syncthreads();
 
   if (live) {
+    p.bias_prev[o] = p.bias[o];
     p.bias[o] = b;
     p.e_prev[o] = e;
     p.loads_last[o] = n;
@@ -139,6 +141,90 @@ __global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlPara
     p.maxvio[layer] = (float)__ddiv_rn(__dsub_rn((double)max_s, nbar), nbar);
     p.minvio[layer] = (float)__ddiv_rn(__dsub_rn(nbar, (double)min_s), nbar);
   }
+}
+
+// Diagnostics the paper plots for the load controller (figure captions of Section 3, Section 4.3), per layer,
+// from the state the last controller update left: out[layer][0] fraction of open worsening gates, [1] share of
+// all assignments that went to the busiest 10 % of the experts (m = round(E/10) experts), [2] fraction of experts
+// without any token, [3] mean |bias change| of the last update.  Integer counts, binary64 ratios rounded once.
+struct DiagParams {
+  int L, E;
+  const int* loads_last;    // [L][E]
+  const int* gate_count;    // [L]
+  const float* bias;        // [L][E]
+  const float* bias_prev;   // [L][E]
+  float* out;               // [L][4]
+};
+
+__global__ void __launch_bounds__(kCtrlThreads) diagnostics_kernel(const DiagParams p) {
+  __shared__ int n_s[kCtrlThreads];
+  __shared__ long long red_a[32], red_b[32];
+  __shared__ int red_c[32];
+  __shared__ double y[kCtrlThreads];
+  const int layer = blockIdx.x, i = threadIdx.x, lane = i & 31, warp = i >> 5;
+  const bool live = i < p.E;
+  const size_t o = (size_t)layer * p.E + i;
+  const int n = live ? p.loads_last[o] : -1;
+  n_s[i] = n;
+  y[i] = live ? fabs((double)p.bias[o] - (double)p.bias_prev[o]) : 0.0;
+  __syncthreads();
+  // rank of expert i by load (descending, ties by index): the m best ranks are the busiest experts
+  int rank = 0;
+  if (live)
+    for (int j = 0; j < p.E; ++j) {
+      const int nj = n_s[j];
+      rank += (nj > n) || (nj == n && j < i);
+    }
+  int m = (p.E + 5) / 10;
+  if (m < 1) m = 1;
+  long long tot = live ? n : 0, top = (live && rank < m) ? n : 0;
+  int empty = (live && n == 0) ? 1 : 0;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    tot += __shfl_xor_sync(0xffffffffu, tot, d);
+    top += __shfl_xor_sync(0xffffffffu, top, d);
+    empty += __shfl_xor_sync(0xffffffffu, empty, d);
+  }
+  if (lane == 0) { red_a[warp] = tot; red_b[warp] = top; red_c[warp] = empty; }
+  for (int stride = kCtrlThreads / 2; stride >= 1; stride >>= 1) {
+    __syncthreads();
+    if (i < stride) y[i] = __dadd_rn(y[i], y[i + stride]);
+  }
+  __syncthreads();
+  if (i == 0) {
+    long long t = 0, tp = 0;
+    int em = 0;
+    for (int w = 0; w < kCtrlThreads / 32; ++w) { t += red_a[w]; tp += red_b[w]; em += red_c[w]; }
+    float* out = p.out + (size_t)layer * 4;
+    out[0] = (float)__ddiv_rn((double)p.gate_count[layer], (double)p.E);
+    out[1] = t > 0 ? (float)__ddiv_rn((double)tp, (double)t) : 0.0f;
+    out[2] = (float)__ddiv_rn((double)em, (double)p.E);
+    out[3] = (float)__ddiv_rn(y[0], (double)p.E);
+  }
+}
+
+// Mean over tokens of the top-K gating-score entropy H = -sum_k w_k ln w_k (nats, Section 4.3), one CTA per
+// layer, binary64 with a fixed summation order (per thread: tokens tid, tid+1024, ...; then a pairwise tree).
+__global__ void __launch_bounds__(kCtrlThreads) gate_entropy_kernel(const float* gate, int T, int K, float* out) {
+  __shared__ double y[kCtrlThreads];
+  const int layer = blockIdx.x, i = threadIdx.x;
+  const float* g = gate + (size_t)layer * T * K;
+  double acc = 0.0;
+  for (int t = i; t < T; t += kCtrlThreads) {
+    double h = 0.0;
+    for (int k = 0; k < K; ++k) {
+      const double w = (double)g[(size_t)t * K + k];
+      if (w > 0.0) h -= w * log(w);
+    }
+    acc += h;
+  }
+  y[i] = acc;
+  for (int stride = kCtrlThreads / 2; stride >= 1; stride >>= 1) {
+    __syncthreads();
+    if (i < stride) y[i] = y[i] + y[i + stride];
+  }
+  __syncthreads();
+  if (i == 0) out[layer] = (float)(y[0] / (double)T);
 }
 
 // loads_acc[i] += add[i]

@@ -24,7 +24,7 @@ constexpr size_t kAlign = 256;
 constexpr size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-  size_t status, bias, e_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
+  size_t status, bias, e_prev, bias_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
   size_t qb_target, qb_hist, qb_prefix, qb_rank;
   size_t state_end;  // everything before this is cleared at init
   size_t stage_x, stage_w, stage_idx, stage_gate;
@@ -39,6 +39,7 @@ Layout make_layout(const moe_route_config& c) {
   l.status = take(64);
   l.bias = take(LE * 4);
   l.e_prev = take(LE * 4);
+  l.bias_prev = take(LE * 4);
   l.loads_acc = take(LE * 4);
   l.loads_last = take(LE * 4);
   l.maxvio = take((size_t)c.num_layers * 4);
@@ -352,6 +353,7 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
   p.ki = c.ki; p.kd = c.kd; p.eta = c.eta; p.rho = c.qb_ema_rho; p.center = ctx->center_on;
   p.bias = at<float>(ctx, ctx->lay.bias);
   p.e_prev = at<float>(ctx, ctx->lay.e_prev);
+  p.bias_prev = at<float>(ctx, ctx->lay.bias_prev);
   p.loads_acc = at<int>(ctx, ctx->lay.loads_acc);
   p.loads_last = at<int>(ctx, ctx->lay.loads_last);
   p.maxvio = at<float>(ctx, ctx->lay.maxvio);
@@ -405,6 +407,38 @@ int moe_gate_stats(moe_route_ctx* ctx, int32_t* gate_count, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   ctx->last_stream = st;
   return copy_out(ctx, gate_count, ctx->lay.gate_count, (size_t)ctx->cfg.num_layers * 4, st);
+}
+
+int moe_load_diagnostics(moe_route_ctx* ctx, float* diag, void* cuda_stream) {
+  if (!ctx || !diag) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  DiagParams d{};
+  d.L = ctx->cfg.num_layers; d.E = ctx->cfg.num_experts;
+  d.loads_last = at<int>(ctx, ctx->lay.loads_last);
+  d.gate_count = at<int>(ctx, ctx->lay.gate_count);
+  d.bias = at<float>(ctx, ctx->lay.bias);
+  d.bias_prev = at<float>(ctx, ctx->lay.bias_prev);
+  d.out = diag;
+  diagnostics_kernel<<<d.L, kCtrlThreads, 0, st>>>(d);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "diagnostics_kernel launch");
+  ctx->launches += 1;
+  return MOE_OK;
+}
+
+int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tokens, float* entropy, void* cuda_stream) {
+  if (!ctx || !topk_gate || !entropy) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (num_tokens < 1) return fail(ctx, MOE_ERR_INVALID_ARG, "num_tokens must be positive");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  gate_entropy_kernel<<<ctx->cfg.num_layers, kCtrlThreads, 0, st>>>(topk_gate, num_tokens, ctx->cfg.top_k, entropy);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "gate_entropy_kernel launch");
+  ctx->launches += 1;
+  return MOE_OK;
 }
 
 int moe_loads_peek(moe_route_ctx* ctx, int32_t* loads, void* cuda_stream) {

@@ -301,6 +301,35 @@ def test_argument_errors_are_reported_not_raised_by_cuda():
     assert r.poll(raise_on_error=False) == binding.MOE_OK
 
 
+def test_diagnostics_match_oracle():
+    # the paper's load-control diagnostics after an ID update, and the gate entropy of a routing step
+    wl = synth.WORKLOADS["tiny_top3"].with_(T=1536, L=2)
+    dev = "cuda"
+    r = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T)
+    w = torch.stack([synth.router_weights(wl, l, dev) for l in range(wl.L)])
+    b_old = np.zeros((wl.L, wl.E), np.float32)
+    ep = np.zeros((wl.L, wl.E), np.float32)
+    for t in range(4):
+        x = torch.stack([synth.hidden_states(wl, l, t, dev) for l in range(wl.L)])
+        idx, gate = r.route_step(x, w)
+        r.controller_update()
+        r.poll()
+        loads, bias, _, _ = [np_(v) for v in r.load_stats()]
+        diag = np_(r.load_diagnostics())
+        ent = np_(r.gate_entropy(gate))
+        for l in range(wl.L):
+            e = oracle.load_error(loads[l].astype(np.int64))
+            b_new, ep[l], g = oracle.id_update(b_old[l], ep[l], e, 6e-3, 6e-3, center=True)
+            np.testing.assert_array_equal(bits(b_new), bits(bias[l]))
+            want = oracle.load_diagnostics(loads[l].astype(np.int64), g, b_old[l], b_new)
+            np.testing.assert_array_equal(bits(diag[l, :3]), bits(want[:3]))      # integer ratios: exact
+            np.testing.assert_allclose(diag[l, 3], want[3], rtol=1e-6)            # fp64 sum, other order
+            np.testing.assert_allclose(ent[l], oracle.gate_entropy_mean(np_(gate)[l]), rtol=1e-6)
+            assert 0 < ent[l] <= np.log(wl.K) + 1e-6
+            b_old[l] = b_new
+    assert diag[:, 1].min() > 0.1            # imbalanced synthetic loads: the busiest 10 % hold more than 10 %
+
+
 # ------------------------------------------------ full-size configurations
 def _full_size(wl, layers, steps=1, sample=192):
     """Full T and H of a configuration (a few layers of it), in the launch
