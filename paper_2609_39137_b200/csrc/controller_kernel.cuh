@@ -46,6 +46,9 @@ __global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlPara
   // launched with programmatic stream serialisation: the block may already be resident while the
   // routing kernel before it drains; nothing of that kernel's output is touched before this returns
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // the next routing kernel may start its prologue and its operand loads now; its epilogue waits for this
+  // grid before it reads the bias or touches the load accumulators
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int layer = blockIdx.x;
   const int i = threadIdx.x;
   const int lane = i & 31, warp = i >> 5;

@@ -163,8 +163,19 @@ int launch_route(moe_route_ctx* ctx, const RouteParams& rp, int grid, cudaStream
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(route_step_kernel)");
     attr_set[ctx->device & 63] = true;
   }
-  route_step_kernel<KL><<<grid, kRouteThreads, smem, st>>>(ctx->tm_x, ctx->tm_w, rp);
-  cudaError_t e = cudaGetLastError();
+  // programmatic stream serialisation: prologue, TMA loads and MMAs may overlap the tail of the kernel
+  // queued before this one; the epilogue waits for that kernel before it reads the bias
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3(grid);
+  lc.blockDim = dim3(kRouteThreads);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &attr;
+  lc.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&lc, route_step_kernel<KL>, ctx->tm_x, ctx->tm_w, rp);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "route_step_kernel launch");
   ctx->launches += 1;
   return MOE_OK;
