@@ -215,6 +215,7 @@ int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, in
   if (need <= 5) return launch_route<5>(ctx, rp, grid, st);
   if (need <= 8) return launch_route<8>(ctx, rp, grid, st);
   if (need <= 10) return launch_route<10>(ctx, rp, grid, st);
+  if (need <= 11) return launch_route<11>(ctx, rp, grid, st);   // Top-10 with the alpha output (quantile controller)
   return launch_route<17>(ctx, rp, grid, st);
 }
 
@@ -348,7 +349,7 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
     q.target = at<float>(ctx, ctx->lay.qb_target);
     qb_init_kernel<<<64, 256, 0, st>>>(q);
     const int col_groups = (c.num_experts + kQbCols - 1) / kQbCols;
-    int splits = (2 * ctx->num_sms + col_groups - 1) / col_groups;
+    int splits = (6 * ctx->num_sms + col_groups - 1) / col_groups;
     const int max_splits = (q.m + 63) / 64;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
@@ -587,7 +588,7 @@ int moe_quantile_target_static(const float* logits, const float* alpha, int32_t 
   // resets prefix and rank before anything is counted
   qb_init_kernel<<<64, 256, 0, st>>>(q);
   const int col_groups = (num_experts + kQbCols - 1) / kQbCols;
-  int splits = (2 * g_static_sms[dev] + col_groups - 1) / col_groups;
+  int splits = (6 * g_static_sms[dev] + col_groups - 1) / col_groups;
   const int max_splits = (num_tokens + 63) / 64;
   if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;

@@ -22,6 +22,7 @@ namespace moe {
 
 constexpr int kQbCols = 32;       // experts per CTA (one per lane)
 constexpr int kQbThreads = 256;   // 8 warps, each takes every 8th row of the CTA's row range
+constexpr int kQbRowsInFlight = 8;
 
 struct QbParams {
   const float* logits;  // [m][E]
@@ -70,12 +71,27 @@ __global__ void __launch_bounds__(kQbThreads) qb_hist_kernel(QbParams p, int pas
   const int rows_per = (p.m + gridDim.y - 1) / gridDim.y;
   const int r0 = blockIdx.y * rows_per;
   const int r1 = min(p.m, r0 + rows_per);
-  for (int i = r0 + warp; i < r1; i += kQbThreads / 32) {
-    if (live) {
-      const float s = sigmoid_score(p.logits[(size_t)i * p.E + col]);
-      const uint32_t key = margin_key(__fsub_rn(s, p.alpha[i]));
-      const bool match = (pass == 0) || (((key ^ pre) >> (shift + 8)) == 0u);
-      if (match) atomicAdd(&h[((key >> shift) & 255u) * kQbCols + lane], 1u);
+  // kQbRowsInFlight independent 128-byte row segments per warp are requested before any is used:
+  // the kernel is bound by memory latency x bytes in flight, not by arithmetic
+  constexpr int kWarps = kQbThreads / 32;
+  for (int i0 = r0 + warp; i0 < r1; i0 += kWarps * kQbRowsInFlight) {
+    float z[kQbRowsInFlight], a[kQbRowsInFlight];
+#pragma unroll
+    for (int u = 0; u < kQbRowsInFlight; ++u) {
+      const int i = i0 + u * kWarps;
+      const bool ok = live && i < r1;
+      z[u] = ok ? __ldg(p.logits + (size_t)i * p.E + col) : 0.0f;
+      a[u] = ok ? __ldg(p.alpha + i) : 0.0f;
+    }
+#pragma unroll
+    for (int u = 0; u < kQbRowsInFlight; ++u) {
+      const int i = i0 + u * kWarps;
+      if (live && i < r1) {
+        const float s = sigmoid_score(z[u]);
+        const uint32_t key = margin_key(__fsub_rn(s, a[u]));
+        const bool match = (pass == 0) || (((key ^ pre) >> (shift + 8)) == 0u);
+        if (match) atomicAdd(&h[((key >> shift) & 255u) * kQbCols + lane], 1u);
+      }
     }
   }
   __syncthreads();
