@@ -166,8 +166,8 @@ int moe_route_poll(moe_route_ctx* ctx);
 /* Validation utility for the candidate filter of moe_route_step: sweeps every
  * finite fp32 logit and writes to dev_result[0] (device, one float) the largest
  * absolute difference between the approximate score used for filtering and the
- * exact score of Section 2.2.  The filter is sound while this stays below the
- * slack compiled into the kernel (2e-6). */
+ * exact score of Section 2.2.  The filter is sound while this stays below half
+ * of the slack compiled into the kernel (1e-5). */
 int moe_debug_score_gap(float* dev_result, void* cuda_stream);
 
 /* Quantile target without any allocation and without a context (the paper has

@@ -94,10 +94,10 @@ def test_route_is_deterministic_and_accumulates_microbatches():
 
 
 def test_candidate_filter_slack_covers_every_fp32_logit():
-    # the approximate score only pre-selects candidates; it must stay within the
-    # compiled slack (absolute part 4e-6, of which half is the budget) of the exact score
+    # the approximate score (one tanh.approx) only pre-selects candidates; over ALL finite fp32 logits it
+    # must stay within half of the slack compiled into the kernel (2e-5) of the exact score
     gap = binding.debug_score_gap()
-    assert 0.0 < gap < 2e-6, gap
+    assert 0.0 < gap < 1e-5, gap
 
 
 # --------------------------------------------------------------- controllers
