@@ -201,6 +201,13 @@ int moe_debug_score_gap(float* dev_result, void* cuda_stream);
 int moe_quantile_target_static(const float* logits, const float* alpha, int32_t num_tokens,
                                int32_t num_experts, int32_t top_k, float* target_out, void* cuda_stream);
 
+/* Validation utility for the bounded device-side waits: launches one warp that
+ * waits, with the same bounded wait the routing kernel uses and the given
+ * iteration bound, on a barrier phase that nothing ever completes.  The wait
+ * gives up, the kernel returns normally, and the next moe_route_poll reports
+ * MOE_ERR_TIMEOUT (wait id 99); the context stays usable. */
+int moe_debug_wait_timeout(moe_route_ctx* ctx, int32_t spin_limit, void* cuda_stream);
+
 /* Number of kernels this context has launched so far. */
 int64_t moe_route_launch_count(const moe_route_ctx* ctx);
 

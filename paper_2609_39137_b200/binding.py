@@ -24,7 +24,7 @@ SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_i
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
            "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static",
-           "moe_load_diagnostics", "moe_gate_entropy"]
+           "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout"]
 
 
 class MoeRouteConfig(C.Structure):
@@ -76,6 +76,7 @@ def load():
     L.moe_last_error.restype = C.c_char_p
     L.moe_route_destroy.argtypes = [vp]
     L.moe_debug_score_gap.argtypes = [vp, vp]
+    L.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
     L.moe_quantile_target_static.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     _lib = L
     return L
@@ -229,6 +230,10 @@ class Router:
         if rc != MOE_OK and raise_on_error:
             raise MoeRouteError(rc, self.lib.moe_last_error(self.h).decode())
         return rc
+
+    def debug_wait_timeout(self, spin_limit=2000):
+        """Launches the bounded-wait probe (a wait nothing satisfies); poll() then reports MOE_ERR_TIMEOUT."""
+        self._check(self.lib.moe_debug_wait_timeout(self.h, spin_limit, _stream()))
 
     def launch_count(self):
         return int(self.lib.moe_route_launch_count(self.h))

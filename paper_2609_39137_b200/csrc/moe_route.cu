@@ -553,6 +553,33 @@ int moe_debug_read_timers(long long* host_out, int reset) {
 }
 #endif
 
+// One warp waits, with the routing kernel's bounded wait, on an mbarrier phase that nothing completes.
+__global__ void wait_timeout_probe_kernel(int* status, uint32_t spin_limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    moe::ptx::mbar_init(moe::ptx::smem_u32(&bar), 1);
+    abort_flag = 0;
+    moe::ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  moe::WaitCtl wc{&abort_flag, status, spin_limit};
+  const bool ok = moe::wait_phase(moe::ptx::smem_u32(&bar), 0u, wc, 99);
+  if (ok && threadIdx.x == 0) status[1] = -1;   // must not happen: nobody arrives on the barrier
+}
+
+int moe_debug_wait_timeout(moe_route_ctx* ctx, int32_t spin_limit, void* cuda_stream) {
+  if (!ctx || spin_limit < 1) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  wait_timeout_probe_kernel<<<1, 32, 0, st>>>(status_ptr(ctx), (uint32_t)spin_limit);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "wait_timeout_probe_kernel launch");
+  ctx->launches += 1;
+  return MOE_OK;
+}
+
 int moe_quantile_target_static(const float* logits, const float* alpha, int32_t num_tokens, int32_t num_experts,
                                int32_t top_k, float* target_out, void* cuda_stream) {
   if (!logits || !alpha || !target_out) return MOE_ERR_INVALID_ARG;

@@ -330,6 +330,21 @@ def test_diagnostics_match_oracle():
     assert diag[:, 1].min() > 0.1            # imbalanced synthetic loads: the busiest 10 % hold more than 10 %
 
 
+def test_bounded_wait_gives_up_and_reports_timeout():
+    # a wait that nothing satisfies runs out after its iteration bound: the kernel returns, the status
+    # word says MOE_ERR_TIMEOUT, and the same context keeps working afterwards
+    T, H, E, K = 256, 128, 768, 10
+    res = route_once(T, H, E, K, seed=3)
+    r = res["r"]
+    r.debug_wait_timeout(spin_limit=2000)
+    assert r.poll(raise_on_error=False) == binding.MOE_ERR_TIMEOUT
+    assert r.poll(raise_on_error=False) == binding.MOE_OK          # sticky status cleared by the poll
+    idx, gate = r.route_step(res["x"], res["w"])
+    r.poll()
+    np.testing.assert_array_equal(np_(idx), res["idx"])
+    np.testing.assert_array_equal(np_(r.loads_peek()), 2 * res["loads"])
+
+
 # ------------------------------------------------ full-size configurations
 def _full_size(wl, layers, steps=1, sample=192):
     """Full T and H of a configuration (a few layers of it), in the launch
