@@ -68,6 +68,9 @@ def lib():
             L.oracle_load_diagnostics.argtypes = [_i64p, _i32p, _f32p, _f32p, _i64, _f32p]
             L.oracle_gate_entropy_mean.argtypes = [_f32p, _i64, _i64]
             L.oracle_gate_entropy_mean.restype = C.c_double
+            L.oracle_full_pool_entropy_mean.argtypes = [_f32p, _f32p, _i64, _i64, C.c_int]
+            L.oracle_full_pool_entropy_mean.restype = C.c_double
+            L.oracle_aux_loss_stats.argtypes = [_f32p, _i64, _i64, _i64p, _f64p, _f64p, _f64p]
             L.oracle_route_tokens_f64.argtypes = [_u16p, _u16p, _f32p, _i64, _i64, _i64, _i64,
                                                   _f64p, _i32p, _f64p, _f64p, _f64p, _i64p]
             _lib = L
@@ -274,6 +277,28 @@ def load_diagnostics(n, gate, b_old, b_new):
                                      n.shape[0], _p(out, _f32p)):
         raise ValueError("empty batch: sum of loads is zero")
     return out
+
+
+def full_pool_entropy_mean(logits, bias=None, kind="biased_sigmoid"):
+    """Mean over tokens of the full-pool selection-score entropy (nats), Section 4.3.
+    kind "biased_sigmoid": p = clamp(sigmoid(z) + b, 0) normalised; kind "softmax": p = softmax(z)."""
+    logits = _arr(logits, np.float32)
+    T, E = logits.shape
+    bias = np.zeros(E, np.float32) if bias is None else _arr(bias, np.float32)
+    k = {"biased_sigmoid": 0, "softmax": 1}[kind]
+    return float(lib().oracle_full_pool_entropy_mean(_p(logits, _f32p), _p(bias, _f32p), T, E, k))
+
+
+def aux_loss_stats(logits, loads):
+    """Eq. 8 forward statistics: (f [E], P [E], sum_i f_i P_i) from logits [T][E] and the loads of the same tokens."""
+    logits = _arr(logits, np.float32)
+    T, E = logits.shape
+    n = _arr(loads, np.int64)
+    f = np.zeros(E, np.float64)
+    P = np.zeros(E, np.float64)
+    aux = np.zeros(1, np.float64)
+    lib().oracle_aux_loss_stats(_p(logits, _f32p), T, E, _p(n, _i64p), _p(f, _f64p), _p(P, _f64p), _p(aux, _f64p))
+    return f, P, float(aux[0])
 
 
 def gate_entropy_mean(gate):

@@ -446,6 +446,80 @@ double oracle_gate_entropy_mean(const float *gate, int64_t T, int64_t K)
 }
 
 /*
+ * Full-pool selection-score entropy of one token (Section 4.3):
+ * H = - sum_e p_e ln p_e in nats (0 ln 0 = 0), where
+ *   kind 0 (bias-controlled methods): p_e = c_e / sum_j c_j with
+ *           c_e = max(sigmoid(z_e) + b_e, 0), the biased score clamped at zero;
+ *   kind 1 (auxiliary loss): p_e = softmax_e(z) = exp(z_e) / sum_j exp(z_j),
+ *           written as the definition (binary64 exp cannot overflow for
+ *           |z| < 700; router logits are far inside).
+ * A token whose clamped scores are all zero has no distribution; H = 0 then.
+ * z : [E] binary32 logits, b : [E] binary32 bias (ignored for kind 1).
+ */
+double oracle_full_pool_entropy(const float *z, const float *b, int64_t E, int kind)
+{
+    double total = 0.0;
+    for (int64_t e = 0; e < E; ++e) {
+        double c;
+        if (kind == 0) {
+            c = oracle_sigmoid_f64((double)z[e]) + (double)b[e];
+            if (c < 0.0) c = 0.0;
+        } else {
+            c = exp((double)z[e]);
+        }
+        total += c;
+    }
+    if (!(total > 0.0)) return 0.0;
+    double h = 0.0;
+    for (int64_t e = 0; e < E; ++e) {
+        double c;
+        if (kind == 0) {
+            c = oracle_sigmoid_f64((double)z[e]) + (double)b[e];
+            if (c < 0.0) c = 0.0;
+        } else {
+            c = exp((double)z[e]);
+        }
+        double p = c / total;
+        if (p > 0.0) h -= p * log(p);
+    }
+    return h;
+}
+
+/* Mean of oracle_full_pool_entropy over the T tokens of z [T][E]. */
+double oracle_full_pool_entropy_mean(const float *z, const float *b, int64_t T, int64_t E, int kind)
+{
+    double sum = 0.0;
+    for (int64_t t = 0; t < T; ++t) sum += oracle_full_pool_entropy(z + t * E, b, E, kind);
+    return sum / (double)T;
+}
+
+/*
+ * Statistics of the auxiliary balancing loss (Eq. 8), forward only:
+ *   f_i = n_i / T          fraction of the T tokens assigned to expert i,
+ *   P_i = (1/T) sum_x softmax_i(W_r x)   mean router probability,
+ *   aux = sum_i f_i P_i    (the coefficient alpha of Eq. 8 is left to the caller).
+ * z : [T][E] binary32 logits, n : [E] counts of the same T tokens.
+ */
+void oracle_aux_loss_stats(const float *z, int64_t T, int64_t E, const int64_t *n,
+                           double *f, double *P, double *aux)
+{
+    for (int64_t e = 0; e < E; ++e) P[e] = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+        const float *zt = z + t * E;
+        double total = 0.0;
+        for (int64_t e = 0; e < E; ++e) total += exp((double)zt[e]);
+        for (int64_t e = 0; e < E; ++e) P[e] += exp((double)zt[e]) / total;
+    }
+    double a = 0.0;
+    for (int64_t e = 0; e < E; ++e) {
+        P[e] /= (double)T;
+        f[e] = (double)n[e] / (double)T;
+        a += f[e] * P[e];
+    }
+    *aux = a;
+}
+
+/*
  * One whole routing pass of the definition for a slice of tokens: logits,
  * scores, biased top-K, gates and load counts (Section 2.2, Algorithm 1
  * lines 3-4).  Convenience for timing and for tests; it only chains the

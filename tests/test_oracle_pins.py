@@ -479,6 +479,76 @@ def test_gate_entropy_closed_forms():
     assert abs(oracle.gate_entropy_mean(w) - ref) < 1e-12
 
 
+def test_full_pool_entropy_closed_forms_and_library():
+    E = 768
+    # equal logits, zero bias: both score families are uniform over the pool, H = ln E
+    z = np.full((5, E), 0.7, np.float32)
+    for kind in ("biased_sigmoid", "softmax"):
+        assert abs(oracle.full_pool_entropy_mean(z, None, kind) - np.log(E)) < 1e-12
+    # softmax entropy ignores a common shift of the logits; it never exceeds ln E
+    rng = np.random.default_rng(72)
+    z = rng.normal(0, 2.0, (40, E)).astype(np.float32)
+    h = oracle.full_pool_entropy_mean(z, None, "softmax")
+    zs = (z.astype(np.float64) + 3.0).astype(np.float32)   # shift representable up to fp32 rounding of z
+    assert abs(oracle.full_pool_entropy_mean(zs, None, "softmax") - h) < 1e-5
+    assert 0.0 < h < np.log(E)
+    # against the library softmax / entropy routines
+    p = scipy.special.softmax(z.astype(np.float64), axis=1)
+    assert abs(h - scipy.special.entr(p).sum(1).mean()) < 1e-12
+    b = rng.normal(0, 0.05, E).astype(np.float32)
+    c = np.maximum(scipy.special.expit(z.astype(np.float64)) + b.astype(np.float64), 0.0)
+    q = c / c.sum(1, keepdims=True)
+    assert abs(oracle.full_pool_entropy_mean(z, b, "biased_sigmoid") - scipy.special.entr(q).sum(1).mean()) < 1e-12
+    # the bias enters the biased-sigmoid family and not the softmax family
+    assert oracle.full_pool_entropy_mean(z, b, "softmax") == h
+    assert oracle.full_pool_entropy_mean(z, b, "biased_sigmoid") != oracle.full_pool_entropy_mean(z, None, "biased_sigmoid")
+    # clamping: experts whose biased score is negative leave the pool; the remaining n equal scores give ln n
+    z = np.zeros((3, E), np.float32)
+    b = np.zeros(E, np.float32)
+    b[100:] = -0.75                      # 0.5 - 0.75 < 0 -> clamped to zero
+    assert abs(oracle.full_pool_entropy_mean(z, b, "biased_sigmoid") - np.log(100)) < 1e-12
+    b[:] = -0.75                         # nothing left: no distribution, H = 0
+    assert oracle.full_pool_entropy_mean(z, b, "biased_sigmoid") == 0.0
+    # two-level distribution: one expert with weight a, the others sharing 1 - a
+    z = np.zeros((1, 8), np.float32)
+    z[0, 0] = np.log(7.0)                # softmax: p0 = 7/14 = 1/2, others 1/14 each
+    want = 0.5 * np.log(2.0) + 0.5 * np.log(14.0)
+    assert abs(oracle.full_pool_entropy_mean(z, None, "softmax") - want) < 1e-7
+
+
+def test_aux_loss_statistics_closed_forms():
+    E, T, K = 64, 208, 4
+    rng = np.random.default_rng(73)
+    z = rng.normal(0, 1.5, (T, E)).astype(np.float32)
+    # perfectly even loads: f_i = K/E for all i, and sum_i P_i = 1, so sum_i f_i P_i = K/E whatever the router says
+    assert (T * K) % E == 0
+    n = np.full(E, (T * K) // E, np.int64)
+    f, P, aux = oracle.aux_loss_stats(z, n)
+    assert abs(P.sum() - 1.0) < 1e-12 and abs(f.sum() - K) < 1e-12
+    np.testing.assert_allclose(P, scipy.special.softmax(z.astype(np.float64), axis=1).mean(0), rtol=1e-12)
+    assert abs(aux - K / E) < 1e-12
+    np.testing.assert_allclose(aux, float((f * P).sum()), rtol=1e-13)
+    # all tokens sent to experts 0..K-1 by a router that is certain of expert 0: f_0 = 1, P_0 ~ 1, aux ~ 1
+    z = np.full((T, E), -30.0, np.float32)
+    z[:, 0] = 30.0
+    n = np.zeros(E, np.int64)
+    n[:K] = T
+    f, P, aux = oracle.aux_loss_stats(z, n)
+    assert f[0] == 1.0 and abs(P[0] - 1.0) < 1e-12 and abs(aux - 1.0) < 1e-12
+    # uniform router, any loads: P_i = 1/E, aux = (1/E) sum_i f_i = K/E
+    z = np.zeros((T, E), np.float32)
+    n = rng.multinomial(T * K, np.ones(E) / E).astype(np.int64)
+    f, P, aux = oracle.aux_loss_stats(z, n)
+    np.testing.assert_allclose(P, 1.0 / E, rtol=1e-13)
+    assert abs(aux - K / E) < 1e-12
+    # the loss grows when load and probability concentrate on the same experts (what Eq. 8 penalises)
+    z = rng.normal(0, 1.0, (T, E)).astype(np.float32)
+    z[:, :4] += 3.0
+    hot = np.zeros(E, np.int64); hot[:4] = T
+    cold = np.zeros(E, np.int64); cold[-4:] = T
+    assert oracle.aux_loss_stats(z, hot)[2] > oracle.aux_loss_stats(z, cold)[2]
+
+
 # ------------------------------------------------------------- whole chain
 def test_route_tokens_chain_and_threads_agree():
     from paper_2609_39137_b200 import synth
