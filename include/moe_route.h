@@ -149,6 +149,29 @@ int moe_load_diagnostics(moe_route_ctx* ctx, float* diag, void* cuda_stream);
 int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tokens, float* entropy,
                      void* cuda_stream);
 
+/* Statistics of the router's score distribution over a dumped logit matrix
+ * (`logits` [L][num_tokens][E] fp32 device, as written by moe_route_step's
+ * logits_out), one value per layer, means over the num_tokens tokens:
+ *   entropy_biased  [L]  full-pool selection-score entropy (Section 4.3) of the
+ *                        bias-controlled score family: p_e = max(sigmoid(z_e) + b_e, 0)
+ *                        normalised over the E experts, H = -sum_e p_e ln p_e in nats
+ *                        (b = the context's CURRENT bias: call before the controller
+ *                        update to get the bias the step was routed with; a token whose
+ *                        clamped scores are all zero counts H = 0);
+ *   entropy_softmax [L]  the same entropy for p = softmax(z), the auxiliary-loss family;
+ *   mean_prob    [L][E]  P_i of Eq. 8: mean softmax probability of expert i;
+ *   aux             [L]  sum_i f_i P_i of Eq. 8 with f_i = loads[l][i] / num_tokens (the
+ *                        coefficient alpha is left to the caller); needs `loads`
+ *                        ([L][E] int32 device, the counts of the SAME tokens, e.g. from
+ *                        moe_loads_peek after a single routing step).
+ * Every output pointer may be NULL (that quantity is skipped); all are device memory.
+ * fp32 arithmetic per token, binary64 fixed-order sums across tokens: results are
+ * deterministic; they agree with the binary64 definition to about 1e-6 relative.
+ * Forward statistics only: the gradient side of the auxiliary loss is a training-loop
+ * matter.  Errors: MOE_ERR_INVALID_ARG (null logits, num_tokens < 1, aux without loads). */
+int moe_score_stats(moe_route_ctx* ctx, const float* logits, int32_t num_tokens, const int32_t* loads,
+                    float* entropy_biased, float* entropy_softmax, float* mean_prob, float* aux, void* cuda_stream);
+
 /* Load accumulators not yet consumed: read them, or add external counts
  * (Algorithm 1 line 4: counts are summed over microbatches and the
  * data-parallel group -- a caller that shards tokens adds its peers' counts). */

@@ -24,7 +24,7 @@ SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_i
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
            "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static",
-           "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout"]
+           "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout", "moe_score_stats"]
 
 
 class MoeRouteConfig(C.Structure):
@@ -77,6 +77,7 @@ def load():
     L.moe_route_destroy.argtypes = [vp]
     L.moe_debug_score_gap.argtypes = [vp, vp]
     L.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
+    L.moe_score_stats.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.moe_quantile_target_static.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     _lib = L
     return L
@@ -204,6 +205,24 @@ class Router:
         h = torch.empty(self.L, dtype=torch.float32, device=self.device)
         self._check(self.lib.moe_gate_entropy(self.h, _ptr(topk_gate), T, _ptr(h), _stream()))
         return h
+
+    def score_stats(self, logits, loads=None):
+        """Score-distribution statistics of a dumped logit tensor [L][T][E]: dict of entropy_biased [L],
+        entropy_softmax [L], mean_prob [L][E] and, when `loads` ([L][E] int32 of the same tokens) is given, aux [L]."""
+        T = logits.shape[-2]
+        assert logits.dtype == torch.float32 and logits.is_contiguous() and logits.numel() == self.L * T * self.E
+        if loads is not None:
+            assert loads.dtype == torch.int32 and loads.is_contiguous() and loads.numel() == self.L * self.E
+        out = dict(entropy_biased=torch.empty(self.L, dtype=torch.float32, device=self.device),
+                   entropy_softmax=torch.empty(self.L, dtype=torch.float32, device=self.device),
+                   mean_prob=torch.empty(self.L, self.E, dtype=torch.float32, device=self.device))
+        if loads is not None:
+            out["aux"] = torch.empty(self.L, dtype=torch.float32, device=self.device)
+        self._check(self.lib.moe_score_stats(self.h, _ptr(logits), T, _ptr(loads) if loads is not None else None,
+                                             _ptr(out["entropy_biased"]), _ptr(out["entropy_softmax"]),
+                                             _ptr(out["mean_prob"]), _ptr(out["aux"]) if loads is not None else None,
+                                             _stream()))
+        return out
 
     def loads_peek(self):
         loads = torch.empty(self.L, self.E, dtype=torch.int32, device=self.device)

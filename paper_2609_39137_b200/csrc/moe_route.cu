@@ -14,6 +14,7 @@
 
 #include "controller_kernel.cuh"
 #include "quantile_kernel.cuh"
+#include "score_stats_kernel.cuh"
 #include "route_kernel.cuh"
 
 namespace {
@@ -27,6 +28,7 @@ struct Layout {
   size_t status, bias, e_prev, bias_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
   size_t qb_target, qb_hist, qb_prefix, qb_rank;
   size_t state_end;  // everything before this is cleared at init
+  size_t stat_P, stat_H, stat_aux;   // per-CTA partial sums of moe_score_stats (written before they are read)
   size_t stage_x, stage_w, stage_idx, stage_gate;
   size_t total;
 };
@@ -52,6 +54,12 @@ Layout make_layout(const moe_route_config& c) {
     l.qb_rank = take((size_t)c.num_experts * 4);
   }
   l.state_end = o;
+  {
+    const size_t LC = (size_t)c.num_layers * stat_ctas_per_layer(c.num_layers);
+    l.stat_P = take(LC * c.num_experts * 4);
+    l.stat_H = take(LC * 2 * 4);
+    l.stat_aux = take((size_t)c.num_layers * kStatMaxGroups * 8);
+  }
   if (c.host_staging) {
     const size_t LT = (size_t)c.num_layers * c.max_tokens;
     l.stage_x = take(LT * c.hidden * 2);
@@ -450,6 +458,40 @@ int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tok
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "gate_entropy_kernel launch");
   ctx->launches += 1;
+  return MOE_OK;
+}
+
+int moe_score_stats(moe_route_ctx* ctx, const float* logits, int32_t num_tokens, const int32_t* loads,
+                    float* entropy_biased, float* entropy_softmax, float* mean_prob, float* aux, void* cuda_stream) {
+  if (!ctx || !logits) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  if (num_tokens < 1) return fail(ctx, MOE_ERR_INVALID_ARG, "num_tokens must be positive");
+  if (aux && !loads) return fail(ctx, MOE_ERR_INVALID_ARG, "aux needs the loads of the same tokens");
+  const moe_route_config& c = ctx->cfg;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  ctx->last_stream = st;
+  StatParams p{};
+  p.logits = logits;
+  p.bias = at<float>(ctx, ctx->lay.bias);
+  p.L = c.num_layers; p.T = num_tokens; p.E = c.num_experts; p.C = stat_ctas_per_layer(c.num_layers);
+  p.part_P = at<float>(ctx, ctx->lay.stat_P);
+  p.part_H = at<float>(ctx, ctx->lay.stat_H);
+  p.aux_part = at<double>(ctx, ctx->lay.stat_aux);
+  p.loads = loads; p.h_biased = entropy_biased; p.h_softmax = entropy_softmax; p.mean_prob = mean_prob; p.aux = aux;
+  const dim3 grid(p.C, p.L);
+  if (p.E <= 256) score_stats_kernel<8><<<grid, kStatThreads, 0, st>>>(p);
+  else if (p.E <= 768) score_stats_kernel<24><<<grid, kStatThreads, 0, st>>>(p);
+  else score_stats_kernel<32><<<grid, kStatThreads, 0, st>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_kernel launch");
+  const int groups = (p.E + kStatFinExperts - 1) / kStatFinExperts;
+  score_stats_finish_kernel<<<dim3(groups, p.L), 1024, 0, st>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_finish_kernel launch");
+  score_stats_scalar_kernel<<<p.L, 32, 0, st>>>(p, groups);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_scalar_kernel launch");
+  ctx->launches += 3;
   return MOE_OK;
 }
 

@@ -330,6 +330,36 @@ def test_diagnostics_match_oracle():
     assert diag[:, 1].min() > 0.1            # imbalanced synthetic loads: the busiest 10 % hold more than 10 %
 
 
+@pytest.mark.parametrize("L,T,H,E,K", [(1, 1500, 256, 768, 10), (3, 700, 128, 256, 8), (2, 333, 128, 1024, 5), (1, 40, 64, 72, 3)])
+def test_score_stats_match_oracle(L, T, H, E, K):
+    # full-pool entropies (Section 4.3) and the forward statistics of the auxiliary loss (Eq. 8) against the
+    # binary64 definition on the GPU's own logit dump; fp32 per-token arithmetic -> relative tolerance 1e-5
+    g = torch.Generator().manual_seed(5)
+    bias = (torch.randn(L, E, generator=g) * 0.2)          # large enough that some biased scores clamp at zero
+    res = route_once(T, H, E, K, L=L, bias=bias, seed=17)
+    r = res["r"]
+    loads = r.loads_peek()
+    st = r.score_stats(torch.from_numpy(res["logits"]).cuda(), loads)
+    r.poll()
+    for l in range(L):
+        z = res["logits"][l]
+        hb = oracle.full_pool_entropy_mean(z, res["bias"][l], "biased_sigmoid")
+        hs = oracle.full_pool_entropy_mean(z, None, "softmax")
+        f, P, aux = oracle.aux_loss_stats(z, res["loads"][l].astype(np.int64))
+        assert abs(float(st["entropy_biased"][l]) - hb) <= 1e-5 * hb
+        assert abs(float(st["entropy_softmax"][l]) - hs) <= 1e-5 * hs
+        np.testing.assert_allclose(np_(st["mean_prob"][l]), P, rtol=1e-5, atol=1e-9)
+        assert abs(float(st["aux"][l]) - aux) <= 1e-5 * aux
+    assert ((1.0 / (1.0 + np.exp(-res["logits"].astype(np.float64))) + res["bias"][:, None, :]) < 0).any()   # clamp exercised
+    # deterministic: same call, same bits; outputs are optional
+    st2 = r.score_stats(torch.from_numpy(res["logits"]).cuda(), loads)
+    for k in st:
+        np.testing.assert_array_equal(bits(np_(st[k])), bits(np_(st2[k])))
+    only = r.score_stats(torch.from_numpy(res["logits"]).cuda())
+    assert "aux" not in only
+    np.testing.assert_array_equal(bits(np_(only["mean_prob"])), bits(np_(st["mean_prob"])))
+
+
 def test_bounded_wait_gives_up_and_reports_timeout():
     # a wait that nothing satisfies runs out after its iteration bound: the kernel returns, the status
     # word says MOE_ERR_TIMEOUT, and the same context keeps working afterwards
