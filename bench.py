@@ -234,6 +234,28 @@ def main():
     route_ms = [a.elapsed_time(b) for a, b in ev.values()]
     loads, bias, maxvio, minvio = router.load_stats()
 
+    # ---- per-call breakdown (after the timed region, not part of `value`): every step bracketed by events, so the
+    # two calls are serialised; median and best step, and the two calls separately
+    n_break = max(3, min(args.steps, 48))
+    bev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_break)]
+    for i in range(n_break):
+        bev[i][0].record()
+        router.route_step(xs[i % ring], w, idx, gate)
+        bev[i][1].record()
+        if dist is not None:
+            dp.allreduce_loads(router, dist)
+        router.controller_update()
+        bev[i][2].record()
+    barrier()
+    router.poll()
+    br_route = sorted(a.elapsed_time(b) for a, b, _ in bev)
+    br_ctrl = sorted(b.elapsed_time(c) for _, b, c in bev)
+    br_step = sorted(a.elapsed_time(c) for a, _, c in bev)
+    breakdown = {"steps": n_break, "serialised": True,
+                 "step_ms_median": statistics.median(br_step), "step_ms_best": br_step[0],
+                 "route_step_ms_median": statistics.median(br_route), "route_step_ms_best": br_route[0],
+                 "controller_update_ms_median": statistics.median(br_ctrl), "controller_update_ms_best": br_ctrl[0]}
+
     # ---- end-to-end: host buffers in, host results out, through moe_route_step_host
     e2e_steps = max(3, min(args.steps, 30))
     rh = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T, controller="id", host_staging=True, device=dev)
@@ -296,8 +318,10 @@ def main():
         if not args.no_cpu_baseline:
             threads = os.cpu_count() or 1
             rate, n_tok, dt = cpu_oracle_rate(wl, threads, args.ref_tokens_per_thread)
+            rate1, n_tok1, dt1 = cpu_oracle_rate(wl, 1, max(64, args.ref_tokens_per_thread // 4))
             cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
-                   "sample": f"{n_tok} of {wl.T} tokens of layer 0, all stages, {dt:.1f} s"}
+                   "sample": f"{n_tok} of {wl.T} tokens of layer 0, all stages, {dt:.1f} s",
+                   "single_thread": {"value": rate1, "sample": f"{n_tok1} tokens, {dt1:.1f} s"}}
         h2d = wl.L * wl.T * wl.H * 2 + wl.L * wl.E * wl.H * 2
         d2h = 2 * wl.L * wl.T * wl.K * 4 + 2 * wl.L * 4
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -310,7 +334,7 @@ def main():
                 "roofline": roofline, "cpu_baseline": cpu,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-                "gpu_launches": int(launches), "clocks": clocks,
+                "gpu_launches": int(launches), "clocks": clocks, "breakdown": breakdown,
                 "last_step": {"maxvio_max": float(maxvio.max()), "minvio_max": float(minvio.max())}}
         print(json.dumps(line), flush=True)
     if dist is not None:
