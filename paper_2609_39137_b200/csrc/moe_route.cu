@@ -582,6 +582,11 @@ int moe_debug_score_gap(float* dev_result, void* cuda_stream) {
 
 #ifdef MOE_KERNEL_TIMERS
 // debug builds only: cycle accounting of the route kernel, 32 counters, optionally reset
+int moe_debug_read_marks(unsigned long long* host_out) {
+  cudaDeviceSynchronize();
+  return cudaMemcpyFromSymbol(host_out, moe::g_route_marks, sizeof(unsigned long long) * 32) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
 int moe_debug_read_timers(long long* host_out, int reset) {
   cudaDeviceSynchronize();
   if (host_out && cudaMemcpyFromSymbol(host_out, moe::g_route_timers, sizeof(long long) * 32) != cudaSuccess)
