@@ -9,6 +9,8 @@ token is one token routed through one router layer.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
   python bench.py --impl reference ...     # the CPU oracle, timed as it stands
+  python bench.py --aux [--workload NAME]  # the calls that are not on the timed path (quantile update, score
+                                           # statistics, diagnostics): microseconds and GB/s of each, own JSON line
 
 Prints ONE JSON line (rank 0).
 """
@@ -136,6 +138,65 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+def run_aux(args, wl):
+    """Times the calls that work on the logits dump (not part of a step): the routing step with the dump, the
+    Quantile Balancing update (single layer), the score statistics, and the small diagnostics calls."""
+    from paper_2609_39137_b200 import binding
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    L1 = wl.with_(L=1)
+    w = torch.stack([synth.router_weights(L1, 0, dev)]).contiguous()
+    xs = [torch.stack([synth.hidden_states(L1, 0, s, dev)]).contiguous() for s in range(4)]
+    logits = torch.empty(1, wl.T, wl.E, device=dev)
+    alpha = torch.empty(1, wl.T, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than L2
+
+    def timed(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return statistics.median(ts), min(ts)
+
+    reps = max(3, min(args.steps, 20))
+    out = {}
+    dump_bytes = wl.T * wl.E * 4
+    rq = binding.Router(1, wl.E, wl.K, wl.H, wl.T, controller="quantile", device=dev)
+    state = {"i": 0}
+
+    def qb_route():
+        rq.route_step(xs[state["i"] % 4], w, logits_out=logits, alpha_out=alpha)
+        state["i"] += 1
+    med, best = timed(lambda: (qb_route(), rq.controller_update()), reps)
+    rs = binding.Router(1, wl.E, wl.K, wl.H, wl.T, controller="id", device=dev)
+    r_med, r_best = timed(lambda: rs.route_step(xs[0], w, logits_out=logits, alpha_out=alpha), reps)
+    out["route_step_with_dump_us"] = {"median": r_med, "best": r_best}
+    out["route_plus_quantile_update_us"] = {"median": med, "best": best}
+    out["quantile_update_us"] = {"median": med - r_med, "note": "difference of the two lines above; 4 passes over the dump",
+                                 "dump_GBps": 4 * dump_bytes / max(1e-9, (med - r_med)) / 1e3}
+    rs.controller_update()
+    idx, gate = rs.route_step(xs[0], w, logits_out=logits)
+    loads = rs.loads_peek()
+    med, best = timed(lambda: rs.score_stats(logits, loads), reps)
+    out["score_stats_us"] = {"median": med, "best": best, "dump_GBps": dump_bytes / best / 1e3}
+    med, best = timed(lambda: rs.gate_entropy(gate), reps)
+    out["gate_entropy_us"] = {"median": med, "best": best}
+    rs.controller_update()
+    med, best = timed(lambda: rs.load_diagnostics(), reps)
+    out["load_diagnostics_us"] = {"median": med, "best": best}
+    rs.poll()
+    rq.poll()
+    print(json.dumps({"aux": True, "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "E": wl.E, "K": wl.K, "L": 1},
+                      "l2": "256 MB written between timed calls", "reps": reps, "calls": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -147,6 +208,7 @@ def main():
     ap.add_argument("--ref-tokens-per-thread", type=int, default=1024)
     ap.add_argument("--prewarm-s", type=float, default=0.5, help="untimed seconds of steps before the warm-up")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--aux", action="store_true", help="time the calls outside the step (one GPU) and exit")
     args = ap.parse_args()
 
     wl = synth.WORKLOADS[args.workload]
@@ -154,6 +216,9 @@ def main():
         wl = wl.with_(L=args.layers)
     if args.impl == "reference":
         run_reference(args, wl)
+        return
+    if args.aux:
+        run_aux(args, wl)
         return
 
     from paper_2609_39137_b200 import binding, dp     # fails loudly if the CUDA library is missing

@@ -206,14 +206,21 @@ __global__ void __launch_bounds__(kCtrlThreads) diagnostics_kernel(const DiagPar
   }
 }
 
-// Mean over tokens of the top-K gating-score entropy H = -sum_k w_k ln w_k (nats, Section 4.3), one CTA per
-// layer, binary64 with a fixed summation order (per thread: tokens tid, tid+1024, ...; then a pairwise tree).
-__global__ void __launch_bounds__(kCtrlThreads) gate_entropy_kernel(const float* gate, int T, int K, float* out) {
-  __shared__ double y[kCtrlThreads];
-  const int layer = blockIdx.x, i = threadIdx.x;
+// Mean over tokens of the top-K gating-score entropy H = -sum_k w_k ln w_k (nats, Section 4.3).  Two steps with a
+// fixed summation order, binary64 throughout: grid (kEntropySlices, L) CTAs each sum a contiguous slice of the
+// layer's tokens (per thread: tokens tid, tid+256, ... of the slice; then a pairwise tree) into part[layer][slice];
+// one warp per layer adds the slices in index order.
+constexpr int kEntropySlices = 64;
+constexpr int kEntropyThreads = 256;
+
+__global__ void __launch_bounds__(kEntropyThreads) gate_entropy_kernel(const float* gate, int T, int K, double* part) {
+  __shared__ double y[kEntropyThreads];
+  const int layer = blockIdx.y, slice = blockIdx.x, i = threadIdx.x;
+  const int per = (T + kEntropySlices - 1) / kEntropySlices;
+  const int t0 = slice * per, t1 = min(T, t0 + per);
   const float* g = gate + (size_t)layer * T * K;
   double acc = 0.0;
-  for (int t = i; t < T; t += kCtrlThreads) {
+  for (int t = t0 + i; t < t1; t += kEntropyThreads) {
     double h = 0.0;
     for (int k = 0; k < K; ++k) {
       const double w = (double)g[(size_t)t * K + k];
@@ -222,12 +229,21 @@ __global__ void __launch_bounds__(kCtrlThreads) gate_entropy_kernel(const float*
     acc += h;
   }
   y[i] = acc;
-  for (int stride = kCtrlThreads / 2; stride >= 1; stride >>= 1) {
+  for (int stride = kEntropyThreads / 2; stride >= 1; stride >>= 1) {
     __syncthreads();
     if (i < stride) y[i] = y[i] + y[i + stride];
   }
   __syncthreads();
-  if (i == 0) out[layer] = (float)(y[0] / (double)T);
+  if (i == 0) part[(size_t)layer * kEntropySlices + slice] = y[0];
+}
+
+__global__ void gate_entropy_finish_kernel(const double* part, int T, float* out) {
+  const int layer = blockIdx.x;
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int c = 0; c < kEntropySlices; ++c) s += part[(size_t)layer * kEntropySlices + c];
+    out[layer] = (float)(s / (double)T);
+  }
 }
 
 // loads_acc[i] += add[i]

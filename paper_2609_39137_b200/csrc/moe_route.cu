@@ -26,9 +26,9 @@ constexpr size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign;
 
 struct Layout {
   size_t status, bias, e_prev, bias_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
-  size_t qb_target, qb_hist, qb_prefix, qb_rank;
+  size_t qb_target, qb_hist, qb_prefix, qb_rank, qb_keys;
   size_t state_end;  // everything before this is cleared at init
-  size_t stat_P, stat_H, stat_aux;   // per-CTA partial sums of moe_score_stats (written before they are read)
+  size_t stat_P, stat_H, stat_aux, ent_part;   // per-CTA partial sums of moe_score_stats (written before they are read)
   size_t stage_x, stage_w, stage_idx, stage_gate;
   size_t total;
 };
@@ -54,11 +54,13 @@ Layout make_layout(const moe_route_config& c) {
     l.qb_rank = take((size_t)c.num_experts * 4);
   }
   l.state_end = o;
+  if (c.controller == MOE_CTRL_QUANTILE) l.qb_keys = take((size_t)c.max_tokens * c.num_experts * 4);
   {
     const size_t LC = (size_t)c.num_layers * stat_ctas_per_layer(c.num_layers);
     l.stat_P = take(LC * c.num_experts * 4);
     l.stat_H = take(LC * 2 * 4);
     l.stat_aux = take((size_t)c.num_layers * kStatMaxGroups * 8);
+    l.ent_part = take((size_t)c.num_layers * kEntropySlices * 8);
   }
   if (c.host_staging) {
     const size_t LT = (size_t)c.num_layers * c.max_tokens;
@@ -355,6 +357,7 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
     q.prefix = at<uint32_t>(ctx, ctx->lay.qb_prefix);
     q.rank = at<uint32_t>(ctx, ctx->lay.qb_rank);
     q.target = at<float>(ctx, ctx->lay.qb_target);
+    q.keys = at<uint32_t>(ctx, ctx->lay.qb_keys);
     qb_init_kernel<<<64, 256, 0, st>>>(q);
     const int col_groups = (c.num_experts + kQbCols - 1) / kQbCols;
     int splits = (6 * ctx->num_sms + col_groups - 1) / col_groups;
@@ -454,10 +457,15 @@ int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tok
   if (num_tokens < 1) return fail(ctx, MOE_ERR_INVALID_ARG, "num_tokens must be positive");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   ctx->last_stream = st;
-  gate_entropy_kernel<<<ctx->cfg.num_layers, kCtrlThreads, 0, st>>>(topk_gate, num_tokens, ctx->cfg.top_k, entropy);
+  double* part = at<double>(ctx, ctx->lay.ent_part);
+  gate_entropy_kernel<<<dim3(kEntropySlices, ctx->cfg.num_layers), kEntropyThreads, 0, st>>>(topk_gate, num_tokens,
+                                                                                           ctx->cfg.top_k, part);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "gate_entropy_kernel launch");
-  ctx->launches += 1;
+  gate_entropy_finish_kernel<<<ctx->cfg.num_layers, 32, 0, st>>>(part, num_tokens, entropy);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "gate_entropy_finish_kernel launch");
+  ctx->launches += 2;
   return MOE_OK;
 }
 

@@ -10,8 +10,12 @@
 // shared-memory histogram that is flushed to the global scratch histogram with
 // one atomic per non-empty bin per CTA.  A small scan kernel then fixes the
 // next digit per expert, updates the remaining rank and clears the histogram.
+// With a key scratch (contexts of the quantile controller have one) the first
+// pass stores the 32-bit image of every margin and the three later passes
+// stream those 4 bytes back instead of recomputing the score, which makes them
+// memory-bound instead of instruction-bound.
 //
-// Scratch per context: hist [E][256] u32, prefix [E] u32, rank [E] u32.
+// Scratch per context: hist [E][256] u32, prefix [E] u32, rank [E] u32, keys [max_tokens][E] u32.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -32,6 +36,7 @@ struct QbParams {
   uint32_t* prefix;     // [E] digits fixed so far (high bits)
   uint32_t* rank;       // [E] remaining 1-based rank inside the matching set
   float* target;        // [E] out: Q_j
+  uint32_t* keys;       // [m][E] scratch or null: pass 0 stores every margin's key, later passes read it back
 };
 
 // Monotone map float -> uint32 (a < b as floats  <=>  key(a) < key(b)); -0 is
@@ -71,26 +76,44 @@ __global__ void __launch_bounds__(kQbThreads) qb_hist_kernel(QbParams p, int pas
   const int rows_per = (p.m + gridDim.y - 1) / gridDim.y;
   const int r0 = blockIdx.y * rows_per;
   const int r1 = min(p.m, r0 + rows_per);
-  // kQbRowsInFlight independent 128-byte row segments per warp are requested before any is used:
-  // the kernel is bound by memory latency x bytes in flight, not by arithmetic
+  // kQbRowsInFlight independent 128-byte row segments per warp are requested before any is used
   constexpr int kWarps = kQbThreads / 32;
-  for (int i0 = r0 + warp; i0 < r1; i0 += kWarps * kQbRowsInFlight) {
-    float z[kQbRowsInFlight], a[kQbRowsInFlight];
+  if (p.keys != nullptr && pass > 0) {
+    // keys of pass 0 are read back: no score arithmetic, the pass is a plain stream over 4 bytes per margin
+    for (int i0 = r0 + warp; i0 < r1; i0 += kWarps * kQbRowsInFlight) {
+      uint32_t key[kQbRowsInFlight];
 #pragma unroll
-    for (int u = 0; u < kQbRowsInFlight; ++u) {
-      const int i = i0 + u * kWarps;
-      const bool ok = live && i < r1;
-      z[u] = ok ? __ldg(p.logits + (size_t)i * p.E + col) : 0.0f;
-      a[u] = ok ? __ldg(p.alpha + i) : 0.0f;
+      for (int u = 0; u < kQbRowsInFlight; ++u) {
+        const int i = i0 + u * kWarps;
+        key[u] = (live && i < r1) ? __ldg(p.keys + (size_t)i * p.E + col) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < kQbRowsInFlight; ++u) {
+        const int i = i0 + u * kWarps;
+        if (live && i < r1 && ((key[u] ^ pre) >> (shift + 8)) == 0u)
+          atomicAdd(&h[((key[u] >> shift) & 255u) * kQbCols + lane], 1u);
+      }
     }
+  } else {
+    for (int i0 = r0 + warp; i0 < r1; i0 += kWarps * kQbRowsInFlight) {
+      float z[kQbRowsInFlight], a[kQbRowsInFlight];
 #pragma unroll
-    for (int u = 0; u < kQbRowsInFlight; ++u) {
-      const int i = i0 + u * kWarps;
-      if (live && i < r1) {
-        const float s = sigmoid_score(z[u]);
-        const uint32_t key = margin_key(__fsub_rn(s, a[u]));
-        const bool match = (pass == 0) || (((key ^ pre) >> (shift + 8)) == 0u);
-        if (match) atomicAdd(&h[((key >> shift) & 255u) * kQbCols + lane], 1u);
+      for (int u = 0; u < kQbRowsInFlight; ++u) {
+        const int i = i0 + u * kWarps;
+        const bool ok = live && i < r1;
+        z[u] = ok ? __ldg(p.logits + (size_t)i * p.E + col) : 0.0f;
+        a[u] = ok ? __ldg(p.alpha + i) : 0.0f;
+      }
+#pragma unroll
+      for (int u = 0; u < kQbRowsInFlight; ++u) {
+        const int i = i0 + u * kWarps;
+        if (live && i < r1) {
+          const float s = sigmoid_score(z[u]);
+          const uint32_t key = margin_key(__fsub_rn(s, a[u]));
+          if (p.keys != nullptr) p.keys[(size_t)i * p.E + col] = key;      // pass 0 only
+          const bool match = (pass == 0) || (((key ^ pre) >> (shift + 8)) == 0u);
+          if (match) atomicAdd(&h[((key >> shift) & 255u) * kQbCols + lane], 1u);
+        }
       }
     }
   }
