@@ -105,7 +105,7 @@ int moe_route_init(const moe_route_config* cfg, void* dev_workspace, size_t work
  * fixed (Algorithm 1 line 3) and ADDS the selections to the per-expert load
  * accumulators (line 4) -- several calls before a controller update are the
  * microbatch case.  logits_out and alpha_out may be NULL.  With
- * MOE_CTRL_QUANTILE both must be given (L must be 1); they are read again by
+ * MOE_CTRL_QUANTILE both must be given; they are read again by
  * the next moe_controller_update and must stay valid until then. */
 int moe_route_step(moe_route_ctx* ctx, const void* x_bf16, const void* w_bf16, int32_t num_tokens,
                    int32_t* topk_idx, float* topk_gate, float* logits_out, float* alpha_out,

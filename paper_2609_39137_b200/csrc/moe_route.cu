@@ -85,7 +85,6 @@ bool config_ok(const moe_route_config* c) {
   if (!(c->qb_ema_rho >= 0.0f) || !(c->qb_ema_rho < 1.0f)) return false;
   if (c->center < -1 || c->center > 1) return false;
   if (c->spin_limit < 0) return false;
-  if (c->controller == MOE_CTRL_QUANTILE && c->num_layers != 1) return false;
   return true;
 }
 
@@ -351,24 +350,33 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
   ctx->last_stream = st;
   if (c.controller == MOE_CTRL_QUANTILE) {
     if (!ctx->qb_logits) return fail(ctx, MOE_ERR_STATE, "quantile controller: no routing step since the last update");
-    QbParams q{};
-    q.logits = ctx->qb_logits; q.alpha = ctx->qb_alpha; q.m = ctx->qb_tokens; q.E = c.num_experts; q.K = c.top_k;
-    q.hist = at<uint32_t>(ctx, ctx->lay.qb_hist);
-    q.prefix = at<uint32_t>(ctx, ctx->lay.qb_prefix);
-    q.rank = at<uint32_t>(ctx, ctx->lay.qb_rank);
-    q.target = at<float>(ctx, ctx->lay.qb_target);
-    q.keys = at<uint32_t>(ctx, ctx->lay.qb_keys);
-    qb_init_kernel<<<64, 256, 0, st>>>(q);
     const int col_groups = (c.num_experts + kQbCols - 1) / kQbCols;
     int splits = (6 * ctx->num_sms + col_groups - 1) / col_groups;
-    const int max_splits = (q.m + 63) / 64;
+    const int max_splits = (ctx->qb_tokens + 63) / 64;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
-    for (int pass = 0; pass < 4; ++pass) {
-      qb_hist_kernel<<<dim3(col_groups, splits), kQbThreads, 0, st>>>(q, pass);
-      qb_scan_kernel<<<(c.num_experts * 32 + 255) / 256, 256, 0, st>>>(q, pass);
+    // Eq. 7 is per layer: the layers take turns on the one radix-select scratch (same stream, so in order)
+    for (int l = 0; l < c.num_layers; ++l) {
+      QbParams q{};
+      q.logits = ctx->qb_logits + (size_t)l * ctx->qb_tokens * c.num_experts;
+      q.alpha = ctx->qb_alpha + (size_t)l * ctx->qb_tokens;
+      q.m = ctx->qb_tokens; q.E = c.num_experts; q.K = c.top_k;
+      q.hist = at<uint32_t>(ctx, ctx->lay.qb_hist);
+      q.prefix = at<uint32_t>(ctx, ctx->lay.qb_prefix);
+      q.rank = at<uint32_t>(ctx, ctx->lay.qb_rank);
+      q.target = at<float>(ctx, ctx->lay.qb_target) + (size_t)l * c.num_experts;
+      q.keys = at<uint32_t>(ctx, ctx->lay.qb_keys);
+      qb_init_kernel<<<64, 256, 0, st>>>(q);
+      for (int pass = 0; pass < 4; ++pass) {
+        qb_hist_kernel<<<dim3(col_groups, splits), kQbThreads, 0, st>>>(q, pass);
+        qb_scan_kernel<<<(c.num_experts * 32 + 255) / 256, 256, 0, st>>>(q, pass);
+      }
+      ctx->launches += 9;
     }
-    ctx->launches += 9;
+    {
+      cudaError_t qe = cudaGetLastError();
+      if (qe != cudaSuccess) return cuda_fail(ctx, qe, "quantile kernels launch");
+    }
     ctx->qb_logits = nullptr;
   }
   CtrlParams p{};
