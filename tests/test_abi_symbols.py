@@ -41,12 +41,16 @@ def test_workspace_bytes_and_config_validation(lib):
     assert lib.moe_route_workspace_bytes(C.byref(cfg)) > n + 48 * 16384 * 2048 * 2
     bad = [dict(num_experts=770), dict(num_experts=2048), dict(top_k=0), dict(top_k=17), dict(hidden=100),
            dict(num_layers=0), dict(max_tokens=0), dict(controller=7), dict(qb_ema_rho=1.0), dict(ki=-1.0),
-           dict(struct_size=8), dict(controller=binding.MOE_CTRL_QUANTILE)]   # quantile needs L == 1
+           dict(struct_size=8)]
     for kw in bad:
         c = binding.default_config(48, 768, 10, 2048, 16384)
         for k, v in kw.items():
             setattr(c, k, v)
         assert lib.moe_route_workspace_bytes(C.byref(c)) == 0, kw
+    # the quantile controller adds its radix-select scratch (histogram + one key per margin of a layer)
+    cq = binding.default_config(48, 768, 10, 2048, 16384)
+    cq.controller = binding.MOE_CTRL_QUANTILE
+    assert lib.moe_route_workspace_bytes(C.byref(cq)) >= n + 16384 * 768 * 4 + 768 * 256 * 4
     h = C.c_void_p()
     c = binding.default_config(1, 768, 10, 2048, 128)
     assert lib.moe_route_init(C.byref(c), None, 0, C.byref(h)) == binding.MOE_ERR_WORKSPACE
