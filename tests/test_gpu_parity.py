@@ -365,6 +365,39 @@ def test_score_stats_match_oracle(L, T, H, E, K):
     np.testing.assert_array_equal(bits(np_(only["mean_prob"])), bits(np_(st["mean_prob"])))
 
 
+def test_step_replays_from_a_cuda_graph():
+    # routing + controller update captured once into a CUDA graph (both launches use programmatic stream
+    # serialisation) and replayed: state and outputs evolve exactly as with eager launches
+    T, H, E, K, L = 640, 256, 768, 10, 2
+    g = torch.Generator(device="cuda").manual_seed(77)
+    x = torch.randn(L, T, H, device="cuda", generator=g).to(torch.bfloat16)
+    w = (torch.randn(L, E, H, device="cuda", generator=g) / 16).to(torch.bfloat16)
+    eager = binding.Router(L, E, K, H, T)
+    graphed = binding.Router(L, E, K, H, T)
+    idx_e = torch.empty(L, T, K, dtype=torch.int32, device="cuda")
+    gate_e = torch.empty(L, T, K, device="cuda")
+    idx_g, gate_g = torch.empty_like(idx_e), torch.empty_like(gate_e)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        graphed.route_step(x, w, idx_g, gate_g)
+        graphed.controller_update()
+    for step in range(4):
+        graph.replay()
+        eager.route_step(x, w, idx_e, gate_e)
+        eager.controller_update()
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(np_(idx_g), np_(idx_e))
+        np.testing.assert_array_equal(bits(np_(gate_g)), bits(np_(gate_e)))
+        for a, b in zip(graphed.load_stats(), eager.load_stats()):
+            np.testing.assert_array_equal(bits(np_(a).astype(np.float32)) if a.dtype.is_floating_point else np_(a),
+                                          bits(np_(b).astype(np.float32)) if b.dtype.is_floating_point else np_(b))
+    graphed.poll()
+    eager.poll()
+    assert float(eager.load_stats()[1].abs().max()) > 0          # the bias moved: the replays really updated state
+
+
 def test_bounded_wait_gives_up_and_reports_timeout():
     # a wait that nothing satisfies runs out after its iteration bound: the kernel returns, the status
     # word says MOE_ERR_TIMEOUT, and the same context keeps working afterwards
