@@ -271,9 +271,9 @@ def main():
     barrier()
 
     # ---- timed region: device-resident inputs
-    # the routing launch is bracketed by events on every `stride`-th step only: an event between two kernels
+    # the routing launch is bracketed by events on every `stride`-th step only (16 brackets per run): an event between two kernels
     # keeps the second from overlapping the first one's tail, so most steps run without any
-    stride = 1 if args.steps <= 16 else 8
+    stride = 1 if args.steps <= 16 else max(8, args.steps // 16)
     ev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
           for i in range(0, args.steps, stride)}
     t_all0, t_all1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
