@@ -84,6 +84,10 @@ typedef struct {
                            -1 = per-controller default (ID on, others off) */
   int32_t spin_limit;   /* iteration bound of every device-side wait; 0 = default */
   int32_t host_staging; /* 1 = reserve workspace for moe_route_step_host */
+  int32_t w_layout;     /* layout of the router weights handed to the step calls:
+                           0 = [L][E][H] (W_r in R^{E x d} as Section 2.2 writes it, hidden contiguous),
+                           1 = [L][H][E] (expert contiguous); the library then transposes into
+                           L*E*H*2 bytes of workspace before every routing launch */
 } moe_route_config;
 
 /* Fills *cfg with the paper's defaults (Ki = Kd = 6e-3, eta = 1e-3, rho = 0,
@@ -106,7 +110,12 @@ int moe_route_init(const moe_route_config* cfg, void* dev_workspace, size_t work
  * accumulators (line 4) -- several calls before a controller update are the
  * microbatch case.  logits_out and alpha_out may be NULL.  With
  * MOE_CTRL_QUANTILE both must be given; they are read again by
- * the next moe_controller_update and must stay valid until then. */
+ * the next moe_controller_update and must stay valid until then.
+ * w_bf16 is [L][E][H], or [L][H][E] for contexts made with w_layout = 1.
+ * Ordering: the kernels are enqueued on cuda_stream and may begin (set-up only)
+ * while the work queued before them is still running; they wait for that work
+ * before they read x, W_r, the bias or the accumulators, so x and W_r may be
+ * produced by the kernel queued just before this call. */
 int moe_route_step(moe_route_ctx* ctx, const void* x_bf16, const void* w_bf16, int32_t num_tokens,
                    int32_t* topk_idx, float* topk_gate, float* logits_out, float* alpha_out,
                    void* cuda_stream);

@@ -31,7 +31,8 @@ class MoeRouteConfig(C.Structure):
     _fields_ = [("struct_size", C.c_int32), ("num_layers", C.c_int32), ("num_experts", C.c_int32),
                 ("top_k", C.c_int32), ("hidden", C.c_int32), ("max_tokens", C.c_int32), ("controller", C.c_int32),
                 ("ki", C.c_float), ("kd", C.c_float), ("eta", C.c_float), ("qb_ema_rho", C.c_float),
-                ("center", C.c_int32), ("spin_limit", C.c_int32), ("host_staging", C.c_int32)]
+                ("center", C.c_int32), ("spin_limit", C.c_int32), ("host_staging", C.c_int32),
+                ("w_layout", C.c_int32)]
 
 
 class MoeRouteError(RuntimeError):
@@ -124,7 +125,8 @@ class Router:
     """One routing + load-control context (L layers).  Methods mirror the C entry points."""
 
     def __init__(self, num_layers, num_experts, top_k, hidden, max_tokens, controller="id", ki=None, kd=None,
-                 eta=None, qb_ema_rho=None, center=None, spin_limit=0, host_staging=False, device="cuda"):
+                 eta=None, qb_ema_rho=None, center=None, spin_limit=0, host_staging=False, w_layout=0,
+                 device="cuda"):
         self.lib = load()
         cfg = default_config(num_layers, num_experts, top_k, hidden, max_tokens)
         cfg.controller = CONTROLLERS[controller] if isinstance(controller, str) else int(controller)
@@ -135,6 +137,7 @@ class Router:
         if center is not None: cfg.center = int(center)
         cfg.spin_limit = spin_limit
         cfg.host_staging = int(bool(host_staging))
+        cfg.w_layout = int(w_layout)
         self.cfg = cfg
         self.L, self.E, self.K, self.H, self.max_tokens = num_layers, num_experts, top_k, hidden, max_tokens
         self.device = torch.device(device)

@@ -246,6 +246,26 @@ __global__ void gate_entropy_finish_kernel(const double* part, int T, float* out
   }
 }
 
+// Router weights given expert-contiguous, in [L][H][E] bf16 -> out [L][E][H] (hidden contiguous, the layout the
+// routing kernel's tensor maps describe).  64 x 64 tiles through shared memory; grid (ceil(E/64), ceil(H/64), L),
+// 256 threads; reads and writes are 128-byte rows.
+__global__ void __launch_bounds__(256) transpose_w_kernel(const uint16_t* in, uint16_t* out, int H, int E) {
+  __shared__ uint16_t tile[64][66];
+  const int layer = blockIdx.z, e0 = blockIdx.x * 64, h0 = blockIdx.y * 64;
+  const uint16_t* src = in + (size_t)layer * H * E;
+  uint16_t* dst = out + (size_t)layer * E * H;
+  const int c = threadIdx.x & 63, r4 = threadIdx.x >> 6;
+  for (int r = r4; r < 64; r += 4) {
+    const int h = h0 + r, e = e0 + c;
+    tile[r][c] = (h < H && e < E) ? src[(size_t)h * E + e] : (uint16_t)0;
+  }
+  __syncthreads();
+  for (int r = r4; r < 64; r += 4) {
+    const int e = e0 + r, h = h0 + c;
+    if (e < E && h < H) dst[(size_t)e * H + h] = tile[c][r];
+  }
+}
+
 // loads_acc[i] += add[i]
 __global__ void loads_add_kernel(int* acc, const int* add, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;

@@ -30,6 +30,7 @@ struct Layout {
   size_t state_end;  // everything before this is cleared at init
   size_t stat_P, stat_H, stat_aux, ent_part;   // per-CTA partial sums of moe_score_stats (written before they are read)
   size_t stage_x, stage_w, stage_idx, stage_gate;
+  size_t w_t;   // [L][E][H] bf16 copy of the weights when they are given as [L][H][E]
   size_t total;
 };
 
@@ -69,6 +70,7 @@ Layout make_layout(const moe_route_config& c) {
     l.stage_idx = take(LT * c.top_k * 4);
     l.stage_gate = take(LT * c.top_k * 4);
   }
+  if (c.w_layout == 1) l.w_t = take(LE * c.hidden * 2);
   l.total = o;
   return l;
 }
@@ -85,6 +87,7 @@ bool config_ok(const moe_route_config* c) {
   if (!(c->qb_ema_rho >= 0.0f) || !(c->qb_ema_rho < 1.0f)) return false;
   if (c->center < -1 || c->center > 1) return false;
   if (c->spin_limit < 0) return false;
+  if (c->w_layout != 0 && c->w_layout != 1) return false;
   return true;
 }
 
@@ -193,6 +196,18 @@ int launch_route(moe_route_ctx* ctx, const RouteParams& rp, int grid, cudaStream
 int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, int32_t* idx, float* gate,
                  float* logits, float* alpha, cudaStream_t st) {
   const moe_route_config& c = ctx->cfg;
+  if (c.w_layout == 1) {
+    // expert-contiguous weights: bring them into the layout of the tensor map first (same stream; the routing
+    // kernel's producer waits for the preceding grid before its first load)
+    if (reinterpret_cast<uintptr_t>(w) & 1) return fail(ctx, MOE_ERR_INVALID_ARG, "w must be 2-byte aligned");
+    uint16_t* wt = at<uint16_t>(ctx, ctx->lay.w_t);
+    const dim3 tg((c.num_experts + 63) / 64, (c.hidden + 63) / 64, c.num_layers);
+    transpose_w_kernel<<<tg, 256, 0, st>>>(static_cast<const uint16_t*>(w), wt, c.hidden, c.num_experts);
+    cudaError_t te = cudaGetLastError();
+    if (te != cudaSuccess) return cuda_fail(ctx, te, "transpose_w_kernel launch");
+    ctx->launches += 1;
+    w = wt;
+  }
   if (ctx->map_x_ptr != x || ctx->map_w_ptr != w || ctx->map_tokens != T) {
     if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(w) & 15))
       return fail(ctx, MOE_ERR_INVALID_ARG, "x and w must be 16-byte aligned");
@@ -250,6 +265,7 @@ void moe_route_default_config(moe_route_config* cfg, int32_t num_layers, int32_t
   cfg->center = -1;
   cfg->spin_limit = 0;
   cfg->host_staging = 0;
+  cfg->w_layout = 0;
 }
 
 size_t moe_route_workspace_bytes(const moe_route_config* cfg) {

@@ -365,6 +365,29 @@ def test_score_stats_match_oracle(L, T, H, E, K):
     np.testing.assert_array_equal(bits(np_(only["mean_prob"])), bits(np_(st["mean_prob"])))
 
 
+@pytest.mark.parametrize("T,H,E,K,L", [(300, 192, 768, 10, 2), (130, 72, 40, 3, 1), (257, 320, 256, 8, 3)])
+def test_expert_contiguous_weight_layout(T, H, E, K, L):
+    # weights handed over as [L][H][E]: same results, bit for bit, as with the paper's [L][E][H], and parity with the oracle
+    res = route_once(T, H, E, K, L=L, seed=5)
+    full_check(res, K, rows=np.arange(0, T, 7))
+    wt = res["w"].transpose(1, 2).contiguous()                  # [L][H][E]
+    r = binding.Router(L, E, K, H, T, w_layout=1)
+    logits = torch.empty(L, T, E, device="cuda")
+    idx, gate = r.route_step(res["x"], wt, logits_out=logits)
+    r.poll()
+    np.testing.assert_array_equal(np_(idx), res["idx"])
+    np.testing.assert_array_equal(bits(np_(gate)), bits(res["gate"]))
+    np.testing.assert_array_equal(bits(np_(logits)), bits(res["logits"]))
+    np.testing.assert_array_equal(np_(r.loads_peek()), res["loads"])
+    # host-buffer step with the same layout
+    rh = binding.Router(L, E, K, H, T, w_layout=1, host_staging=True)
+    ih = torch.empty(L, T, K, dtype=torch.int32).pin_memory()
+    gh = torch.empty(L, T, K, dtype=torch.float32).pin_memory()
+    rh.route_step_host(res["x"].cpu().pin_memory(), wt.cpu().pin_memory(), ih, gh)
+    rh.poll()
+    np.testing.assert_array_equal(ih.numpy(), res["idx"])
+
+
 def test_step_replays_from_a_cuda_graph():
     # routing + controller update captured once into a CUDA graph (both launches use programmatic stream
     # serialisation) and replayed: state and outputs evolve exactly as with eager launches
