@@ -365,6 +365,38 @@ def test_score_stats_match_oracle(L, T, H, E, K):
     np.testing.assert_array_equal(bits(np_(only["mean_prob"])), bits(np_(st["mean_prob"])))
 
 
+def _fuzz_case(seed):
+    rng = np.random.default_rng(seed)
+    E = int(rng.choice([8, 16, 40, 64, 128, 256, 264, 512, 768, 776, 1000, 1024]))
+    K = int(rng.integers(1, min(16, E - 1) + 1))
+    H = int(rng.choice([8, 16, 64, 72, 128, 200, 256, 320, 512]))
+    T = int(rng.integers(1, 700))
+    L = int(rng.integers(1, 4))
+    bias_scale = float(rng.choice([0.0, 1e-3, 1e-2, 0.3, 2.0]))
+    logit_scale = float(rng.choice([0.05, 1.0, 4.0]))
+    quantise = bool(rng.integers(0, 3) == 0)          # coarse inputs: many exactly equal scores
+    return T, H, E, K, L, bias_scale, logit_scale, quantise
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_route_random_shapes_bit_exact(seed):
+    # seeded random shapes, bias magnitudes, logit spreads and tie densities: the binary32 chain must match the
+    # oracle bit for bit on the GPU's own logits (indices, gates, alpha), and the loads must be the recount
+    T, H, E, K, L, bias_scale, logit_scale, quantise = _fuzz_case(1000 + seed)
+    g = torch.Generator().manual_seed(seed)
+    bias = torch.randn(L, E, generator=g) * bias_scale
+    x = torch.randn(L, T, H, generator=g)
+    w = torch.randn(L, E, H, generator=g) * (logit_scale / max(H, 1) ** 0.5)
+    if quantise:
+        x, w, bias = torch.round(x), torch.round(w * 4) / 4, torch.round(bias * 8) / 8
+    res = route_once(T, H, E, K, L=L, bias=bias, want_alpha=(K < 16), x=x.cuda().to(torch.bfloat16),
+                     w=w.cuda().to(torch.bfloat16))
+    for l in range(L):
+        a = None if res["alpha"] is None else res["alpha"][l]
+        oi = check_exact(res["logits"][l], res["bias"][l], K, res["idx"][l], res["gate"][l], a)
+        np.testing.assert_array_equal(res["loads"][l], np.bincount(oi.ravel(), minlength=E))
+
+
 @pytest.mark.parametrize("T,H,E,K,L", [(300, 192, 768, 10, 2), (130, 72, 40, 3, 1), (257, 320, 256, 8, 3)])
 def test_expert_contiguous_weight_layout(T, H, E, K, L):
     # weights handed over as [L][H][E]: same results, bit for bit, as with the paper's [L][E][H], and parity with the oracle
