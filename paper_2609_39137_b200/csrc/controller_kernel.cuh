@@ -12,6 +12,7 @@
 // strides 512, 256, ..., 1.
 #pragma once
 #include <cuda_runtime.h>
+#include <limits.h>
 #include <stdint.h>
 
 namespace moe {
@@ -36,114 +37,147 @@ struct CtrlParams {
   int* status;
 };
 
-__global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlParams p) {
-  __shared__ double y[kCtrlThreads];
-  __shared__ long long red_sum[32];
-  __shared__ int red_max[32], red_min[32], red_gate[32];
-  __shared__ long long total_s;
-  __shared__ int max_s, min_s;
+// Shared-memory scratch of one controller step.
+struct CtrlScratch {
+  double y[1024];
+  long long red_sum[32];
+  int red_max[32], red_min[32], red_gate[32];
+  long long total_s;
+  int max_s, min_s;
+};
 
-  // launched with programmatic stream serialisation: the block may already be resident while the
-  // routing kernel before it drains; nothing of that kernel's output is touched before this returns
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  // the next routing kernel may start its prologue and its operand loads now; its epilogue waits for this
-  // grid before it reads the bias or touches the load accumulators
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const int layer = blockIdx.x;
-  const int i = threadIdx.x;
-  const int lane = i & 31, warp = i >> 5;
-  const bool live = i < p.E;
-  const size_t o = (size_t)layer * p.E + i;
-
-  const int n = live ? p.loads_acc[o] : 0;
-  long long s = n;
-  int mx = live ? n : INT_MIN;
-  int mn = live ? n : INT_MAX;
+// One controller step of one layer by NT threads (NT = 1024: one expert per thread; NT = 256: four), tid in
+// [0, NT).  `sync` is a barrier over exactly these NT threads.  The integer reductions are order-free; the
+// centring sum keeps its fixed order (y[i] += y[i + stride], strides 512 ... 1) for any NT.  Loads are read
+// from L2 (they were accumulated there with atomics, possibly by other CTAs of the same launch).
+template <int NT, typename Sync>
+__device__ __forceinline__ void controller_layer(const CtrlParams& p, int layer, int tid, CtrlScratch* sc, Sync sync) {
+  constexpr int PER = 1024 / NT;
+  const int lane = tid & 31, warp = tid >> 5;
+  int n[PER];
+  long long s = 0;
+  int mx = INT_MIN, mn = INT_MAX;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int i = tid + j * NT;
+    const bool live = i < p.E;
+    n[j] = live ? __ldcg(p.loads_acc + (size_t)layer * p.E + i) : 0;
+    s += n[j];
+    mx = max(mx, live ? n[j] : INT_MIN);
+    mn = min(mn, live ? n[j] : INT_MAX);
+  }
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) {
     s += __shfl_xor_sync(0xffffffffu, s, d);
     mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, d));
     mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, d));
   }
-  if (lane == 0) { red_sum[warp] = s; red_max[warp] = mx; red_min[warp] = mn; }
-  __syncthreads();
+  if (lane == 0) { sc->red_sum[warp] = s; sc->red_max[warp] = mx; sc->red_min[warp] = mn; }
+  sync();
   if (warp == 0) {
-    s = red_sum[lane]; mx = red_max[lane]; mn = red_min[lane];
+    const bool has = lane < NT / 32;
+    s = has ? sc->red_sum[lane] : 0; mx = has ? sc->red_max[lane] : INT_MIN; mn = has ? sc->red_min[lane] : INT_MAX;
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
       s += __shfl_xor_sync(0xffffffffu, s, d);
       mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, d));
       mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, d));
     }
-    if (lane == 0) { total_s = s; max_s = mx; min_s = mn; }
+    if (lane == 0) { sc->total_s = s; sc->max_s = mx; sc->min_s = mn; }
   }
-  __syncthreads();
-  const long long total = total_s;
+  sync();
+  const long long total = sc->total_s;
   if (total <= 0) {
     // empty batch: the error of Eq. 3 is undefined; leave the layer untouched
-    if (i == 0) atomicCAS(p.status, 0, kStatusState);
+    if (tid == 0) atomicCAS(p.status, 0, kStatusState);
     return;
   }
   const double nbar = __ddiv_rn((double)total, (double)p.E);
-  const float e = live ? (float)__ddiv_rn(__dsub_rn(nbar, (double)n), nbar) : 0.0f;
-
-  float b = live ? p.bias[o] : 0.0f;
-  const float ep = live ? p.e_prev[o] : 0.0f;
-  int gate = 0;
-  if (p.controller == 0) {                       // ID Balancing
-    const float de = __fsub_rn(e, ep);
-    gate = ((ep > 0.0f && de > 0.0f) || (ep < 0.0f && de < 0.0f)) ? 1 : 0;
-    const float t1 = __fmul_rn(p.ki, e);
-    const float t2 = gate ? __fmul_rn(p.kd, de) : 0.0f;
-    b = __fadd_rn(__fadd_rn(b, t1), t2);
-  } else if (p.controller == 1) {                // fixed-step integral
-    const float step = (e > 0.0f) ? p.eta : (e < 0.0f) ? -p.eta : 0.0f;
-    b = __fadd_rn(b, step);
-  } else if (p.controller == 2) {                // quantile target (+ EMA)
-    const float q = live ? p.qb_target[o] : 0.0f;
-    if (p.rho == 0.0f) {
-      b = q;
-    } else {
-      const float keep = __fmul_rn(p.rho, b);
-      const float take = __fmul_rn(__fsub_rn(1.0f, p.rho), q);
-      b = __fadd_rn(keep, take);
+  float b[PER], e[PER];
+  int gsum = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int i = tid + j * NT;
+    const bool live = i < p.E;
+    const size_t o = (size_t)layer * p.E + i;
+    e[j] = live ? (float)__ddiv_rn(__dsub_rn(nbar, (double)n[j]), nbar) : 0.0f;
+    b[j] = live ? p.bias[o] : 0.0f;
+    const float ep = live ? p.e_prev[o] : 0.0f;
+    int gate = 0;
+    if (p.controller == 0) {                       // ID Balancing
+      const float de = __fsub_rn(e[j], ep);
+      gate = ((ep > 0.0f && de > 0.0f) || (ep < 0.0f && de < 0.0f)) ? 1 : 0;
+      const float t1 = __fmul_rn(p.ki, e[j]);
+      const float t2 = gate ? __fmul_rn(p.kd, de) : 0.0f;
+      b[j] = __fadd_rn(__fadd_rn(b[j], t1), t2);
+    } else if (p.controller == 1) {                // fixed-step integral
+      const float step = (e[j] > 0.0f) ? p.eta : (e[j] < 0.0f) ? -p.eta : 0.0f;
+      b[j] = __fadd_rn(b[j], step);
+    } else if (p.controller == 2) {                // quantile target (+ EMA)
+      const float q = live ? p.qb_target[o] : 0.0f;
+      if (p.rho == 0.0f) {
+        b[j] = q;
+      } else {
+        const float keep = __fmul_rn(p.rho, b[j]);
+        const float take = __fmul_rn(__fsub_rn(1.0f, p.rho), q);
+        b[j] = __fadd_rn(keep, take);
+      }
     }
+    if (live) gsum += gate;
   }
-  if (!live) gate = 0;
 
   if (p.center) {
-    y[i] = live ? (double)b : 0.0;
-    __syncthreads();
-#pragma unroll 1
-    for (int stride = kCtrlThreads / 2; stride >= 1; stride >>= 1) {
-      // y[i + stride] is not written during this pass, so one barrier suffices
-      if (i < stride) y[i] = __dadd_rn(y[i], y[i + stride]);
-      __syncthreads();
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int i = tid + j * NT;
+      sc->y[i] = (i < p.E) ? (double)b[j] : 0.0;
     }
-    const float mean = (float)__ddiv_rn(y[0], (double)p.E);
-    b = __fsub_rn(b, mean);
+    sync();
+#pragma unroll 1
+    for (int stride = 512; stride >= 1; stride >>= 1) {
+      // y[i + stride] is not written during this pass, so one barrier suffices
+      for (int i = tid; i < stride; i += NT) sc->y[i] = __dadd_rn(sc->y[i], sc->y[i + stride]);
+      sync();
+    }
+    const float mean = (float)__ddiv_rn(sc->y[0], (double)p.E);
+#pragma unroll
+    for (int j = 0; j < PER; ++j) b[j] = __fsub_rn(b[j], mean);
   }
 
-  int gsum = gate;
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) gsum += __shfl_xor_sync(0xffffffffu, gsum, d);
-  if (lane == 0) red_gate[warp] = gsum;
-  __syncthreads();
+  if (lane == 0) sc->red_gate[warp] = gsum;
+  sync();
 
-  if (live) {
-    p.bias_prev[o] = p.bias[o];
-    p.bias[o] = b;
-    p.e_prev[o] = e;
-    p.loads_last[o] = n;
-    p.loads_acc[o] = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int i = tid + j * NT;
+    if (i < p.E) {
+      const size_t o = (size_t)layer * p.E + i;
+      p.bias_prev[o] = p.bias[o];
+      p.bias[o] = b[j];
+      p.e_prev[o] = e[j];
+      p.loads_last[o] = n[j];
+      p.loads_acc[o] = 0;
+    }
   }
-  if (i == 0) {
+  if (tid == 0) {
     int gtot = 0;
-    for (int w = 0; w < kCtrlThreads / 32; ++w) gtot += red_gate[w];
+    for (int w = 0; w < NT / 32; ++w) gtot += sc->red_gate[w];
     p.gate_count[layer] = gtot;
-    p.maxvio[layer] = (float)__ddiv_rn(__dsub_rn((double)max_s, nbar), nbar);
-    p.minvio[layer] = (float)__ddiv_rn(__dsub_rn(nbar, (double)min_s), nbar);
+    p.maxvio[layer] = (float)__ddiv_rn(__dsub_rn((double)sc->max_s, nbar), nbar);
+    p.minvio[layer] = (float)__ddiv_rn(__dsub_rn(nbar, (double)sc->min_s), nbar);
   }
+}
+
+__global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlParams p) {
+  __shared__ CtrlScratch sc;
+  // launched with programmatic stream serialisation: the block may already be resident while the
+  // routing kernel before it drains; nothing of that kernel's output is touched before this returns
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // the next routing kernel may be scheduled now; it waits for this grid before it reads anything
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  controller_layer<kCtrlThreads>(p, blockIdx.x, threadIdx.x, &sc, [] { __syncthreads(); });
 }
 
 // Diagnostics the paper plots for the load controller (figure captions of Section 3, Section 4.3), per layer,
