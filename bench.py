@@ -38,7 +38,7 @@ RING = 8   # distinct input batches cycled through, so every timed step reads x 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one route_step_kernel launch, from an ncu capture of
 # this command on the same workload (the summary is kept with the other profile summaries); None = no capture
-NCU_TRAFFIC_BYTES = {"top10_single": 70669568 + 1626368}
+NCU_TRAFFIC_BYTES = {"top10_single": 70629376 + 1660928}
 
 
 def peaks():
