@@ -223,7 +223,7 @@ def _closed_loop(wl, kind, steps, check_rows=None, **kw):
                 checked += c
             Q = oracle.quantile_target(lg[l], al[l], wl.K) if kind == "quantile" else None
             b[l], ep[l], g, mx, mn = oracle_controller_step(
-                kind, b[l], ep[l], loads[l], dict(ki=kw.get("ki", 6e-3), kd=kw.get("kd", 6e-3), eta=kw.get("eta", 1e-3)),
+                kind, b[l], ep[l], loads[l], dict(ki=kw.get("ki", 6e-3), kd=kw.get("kd", 6e-3), eta=kw.get("eta", 1e-3), rho=kw.get("qb_ema_rho", 0.0)),
                 center, Q)
             assert bits(mxv[l:l + 1])[0] == bits(np.array([mx]))[0]
         np.testing.assert_array_equal(bits(bias), bits(b))
@@ -246,6 +246,14 @@ def test_closed_loop_three_controllers_reduced(kind, K):
     wl = synth.WORKLOADS["top3_single"].with_(T=2048, H=512, K=K)
     hist = _closed_loop(wl, kind, 6)
     assert all(0 <= mx <= wl.E / K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn in hist)
+
+
+@pytest.mark.parametrize("rho", [0.5, 0.9])
+def test_closed_loop_quantile_with_ema(rho):
+    # Quantile Balancing with the exponential moving average of Section 3: b = rho b + (1 - rho) Q, bit for bit
+    wl = synth.WORKLOADS["top3_single"].with_(T=1024, H=256, K=3)
+    hist = _closed_loop(wl, "quantile", 5, qb_ema_rho=rho)
+    assert all(0 <= mx <= wl.E / wl.K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn in hist)
 
 
 def test_closed_loop_quantile_two_layers():
