@@ -111,6 +111,9 @@ int moe_route_init(const moe_route_config* cfg, void* dev_workspace, size_t work
  * microbatch case.  logits_out and alpha_out may be NULL.  With
  * MOE_CTRL_QUANTILE both must be given; they are read again by
  * the next moe_controller_update and must stay valid until then.
+ * Alignment: x and w 16 bytes (TMA), logits_out 16 bytes (written with vector
+ * stores), topk_idx / topk_gate / alpha_out 4 bytes; anything else returns
+ * MOE_ERR_INVALID_ARG before a kernel is launched.
  * w_bf16 is [L][E][H], or [L][H][E] for contexts made with w_layout = 1.
  * Ordering: the kernels are enqueued on cuda_stream and may begin (set-up only)
  * while the work queued before them is still running; they wait for that work
@@ -174,25 +177,45 @@ int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tok
  *                        ([L][E] int32 device, the counts of the SAME tokens, e.g. from
  *                        moe_loads_peek after a single routing step).
  * Every output pointer may be NULL (that quantity is skipped); all are device memory.
- * fp32 arithmetic per token, binary64 fixed-order sums across tokens: results are
- * deterministic; they agree with the binary64 definition to about 1e-6 relative.
+ * fp32 arithmetic per token; each warp adds its tokens' values in fp32 (a few
+ * hundred to a thousand rows per warp), the per-CTA partial sums are then added
+ * in a fixed order in binary64: results are deterministic and agree with the
+ * binary64 definition to about 1e-5 relative.
  * Forward statistics only: the gradient side of the auxiliary loss is a training-loop
  * matter.  Errors: MOE_ERR_INVALID_ARG (null logits, num_tokens < 1, aux without loads). */
 int moe_score_stats(moe_route_ctx* ctx, const float* logits, int32_t num_tokens, const int32_t* loads,
                     float* entropy_biased, float* entropy_softmax, float* mean_prob, float* aux, void* cuda_stream);
 
-/* Load accumulators not yet consumed: read them, or add external counts
- * (Algorithm 1 line 4: counts are summed over microbatches and the
- * data-parallel group -- a caller that shards tokens adds its peers' counts). */
+/* Load accumulators not yet consumed: read them, or add external counts.
+ * Algorithm 1 line 4 takes n_i over every microbatch and every data-parallel
+ * rank of the iteration: a caller that shards tokens across GPUs brings the
+ * other ranks' counts in before the controller update. */
 int moe_loads_peek(moe_route_ctx* ctx, int32_t* loads, void* cuda_stream);
 int moe_loads_add(moe_route_ctx* ctx, const int32_t* loads, void* cuda_stream);
 
-/* Controller state (b, e_prev of Algorithm 1) for checkpoint / resume. */
-int moe_state_export(moe_route_ctx* ctx, float* bias, float* e_prev, void* cuda_stream);
-int moe_state_import(moe_route_ctx* ctx, const float* bias, const float* e_prev, void* cuda_stream);
+/* Device address of the accumulators themselves ([L][E] int32, inside the
+ * workspace), for a caller that sums them over its data-parallel group IN PLACE
+ * (one all-reduce(SUM) on this buffer between the last moe_route_step and
+ * moe_controller_update, on the same stream, replaces peek + exchange + add).
+ * The address stays valid for the life of the context.  Host call, nothing is
+ * enqueued. */
+int moe_loads_buffer(moe_route_ctx* ctx, int32_t** dev_loads);
+
+/* Controller state of Algorithm 1 for checkpoint / resume: b and e_prev
+ * ([L][E] float32, device, either may be NULL) and the number of controller
+ * updates this context has enqueued so far (`step_host`, HOST memory, may be
+ * NULL; written before the call returns).  Import restores what is given;
+ * step = -1 keeps the context's own counter. */
+int moe_state_export(moe_route_ctx* ctx, float* bias, float* e_prev, int64_t* step_host, void* cuda_stream);
+int moe_state_import(moe_route_ctx* ctx, const float* bias, const float* e_prev, int64_t step, void* cuda_stream);
 
 /* Synchronises the stream of the last call and returns the sticky device
- * status (MOE_OK, MOE_ERR_TIMEOUT, MOE_ERR_STATE, MOE_ERR_CUDA); clears it. */
+ * status (MOE_OK, MOE_ERR_TIMEOUT, MOE_ERR_STATE, MOE_ERR_CUDA); clears it.
+ * After MOE_ERR_TIMEOUT the routing step that gave up is void: its index and
+ * gate outputs are incomplete, and this call has cleared the load accumulators
+ * (including earlier microbatches of the same iteration), so the next
+ * controller update cannot consume a partial histogram.  Bias and previous
+ * error are untouched; route the iteration again or skip it. */
 int moe_route_poll(moe_route_ctx* ctx);
 
 /* Validation utility for the candidate filter of moe_route_step: sweeps every

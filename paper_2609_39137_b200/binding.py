@@ -22,7 +22,7 @@ CONTROLLERS = {"id": MOE_CTRL_ID, "fixed_step": MOE_CTRL_FIXED_STEP, "quantile":
 # every symbol include/moe_route.h declares
 SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_init", "moe_route_step",
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
-           "moe_loads_add", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
+           "moe_loads_add", "moe_loads_buffer", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
            "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static",
            "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout", "moe_score_stats"]
 
@@ -68,8 +68,9 @@ def load():
     L.moe_gate_entropy.argtypes = [vp, vp, i32, vp, vp]
     L.moe_loads_peek.argtypes = [vp, vp, vp]
     L.moe_loads_add.argtypes = [vp, vp, vp]
-    L.moe_state_export.argtypes = [vp, vp, vp, vp]
-    L.moe_state_import.argtypes = [vp, vp, vp, vp]
+    L.moe_loads_buffer.argtypes = [vp, C.POINTER(vp)]
+    L.moe_state_export.argtypes = [vp, vp, vp, C.POINTER(C.c_int64), vp]
+    L.moe_state_import.argtypes = [vp, vp, vp, C.c_int64, vp]
     L.moe_route_poll.argtypes = [vp]
     L.moe_route_launch_count.argtypes = [vp]
     L.moe_route_launch_count.restype = C.c_int64
@@ -236,16 +237,28 @@ class Router:
         assert loads.dtype == torch.int32 and loads.is_contiguous() and loads.numel() == self.L * self.E
         self._check(self.lib.moe_loads_add(self.h, _ptr(loads), _stream()))
 
-    def state_export(self):
+    def loads_view(self):
+        """int32 [L][E] tensor that aliases the load accumulators inside the workspace (moe_loads_buffer):
+        an in-place all-reduce on it, on the current stream, is the data-parallel exchange."""
+        p = C.c_void_p()
+        self._check(self.lib.moe_loads_buffer(self.h, C.byref(p)))
+        off = p.value - self.workspace.data_ptr()
+        n = self.L * self.E * 4
+        assert 0 <= off and off + n <= self.workspace.numel() and off % 4 == 0
+        return self.workspace[off:off + n].view(torch.int32).view(self.L, self.E)
+
+    def state_export(self, with_step=False):
+        """(bias, e_prev) [L][E] float32; with_step=True adds the controller-update counter."""
         bias = torch.empty(self.L, self.E, dtype=torch.float32, device=self.device)
         e_prev = torch.empty(self.L, self.E, dtype=torch.float32, device=self.device)
-        self._check(self.lib.moe_state_export(self.h, _ptr(bias), _ptr(e_prev), _stream()))
-        return bias, e_prev
+        step = C.c_int64(-1)
+        self._check(self.lib.moe_state_export(self.h, _ptr(bias), _ptr(e_prev), C.byref(step), _stream()))
+        return (bias, e_prev, int(step.value)) if with_step else (bias, e_prev)
 
-    def state_import(self, bias=None, e_prev=None):
+    def state_import(self, bias=None, e_prev=None, step=-1):
         for t in (bias, e_prev):
             assert t is None or (t.dtype == torch.float32 and t.is_contiguous() and t.numel() == self.L * self.E)
-        self._check(self.lib.moe_state_import(self.h, _ptr(bias), _ptr(e_prev), _stream()))
+        self._check(self.lib.moe_state_import(self.h, _ptr(bias), _ptr(e_prev), int(step), _stream()))
 
     def poll(self, raise_on_error=True):
         rc = self.lib.moe_route_poll(self.h)

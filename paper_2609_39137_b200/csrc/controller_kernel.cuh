@@ -46,12 +46,13 @@ struct CtrlScratch {
   int max_s, min_s;
 };
 
-// One controller step of one layer by NT threads (NT = 1024: one expert per thread; NT = 256: four), tid in
-// [0, NT).  `sync` is a barrier over exactly these NT threads.  The integer reductions are order-free; the
-// centring sum keeps its fixed order (y[i] += y[i + stride], strides 512 ... 1) for any NT.  Loads are read
-// from L2 (they were accumulated there with atomics, possibly by other CTAs of the same launch).
-template <int NT, typename Sync>
+// One controller step of one layer by the CTA's 1024 threads, one expert per thread, tid in [0, 1024).  `sync`
+// is a barrier over exactly these threads.  The integer reductions are order-free; the centring sum has a
+// fixed order (y[i] += y[i + stride], strides 512 ... 1).  Loads are read from L2 (they were accumulated
+// there with atomics by the routing kernel's CTAs).
+template <typename Sync>
 __device__ __forceinline__ void controller_layer(const CtrlParams& p, int layer, int tid, CtrlScratch* sc, Sync sync) {
+  constexpr int NT = kCtrlThreads;
   constexpr int PER = 1024 / NT;
   const int lane = tid & 31, warp = tid >> 5;
   int n[PER];
@@ -177,7 +178,7 @@ __global__ void __launch_bounds__(kCtrlThreads) controller_kernel(const CtrlPara
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // the next routing kernel may be scheduled now; it waits for this grid before it reads anything
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  controller_layer<kCtrlThreads>(p, blockIdx.x, threadIdx.x, &sc, [] { __syncthreads(); });
+  controller_layer(p, blockIdx.x, threadIdx.x, &sc, [] { __syncthreads(); });
 }
 
 // Diagnostics the paper plots for the load controller (figure captions of Section 3, Section 4.3), per layer,

@@ -117,6 +117,7 @@ struct moe_route_ctx {
   EncodeTiledFn encode;
   cudaStream_t last_stream;
   int64_t launches;
+  int64_t ctrl_steps;   // controller updates enqueued so far (exported / restored with the controller state)
   // cached TMA descriptors
   const void* map_x_ptr;
   const void* map_w_ptr;
@@ -312,6 +313,12 @@ int moe_route_step(moe_route_ctx* ctx, const void* x_bf16, const void* w_bf16, i
   if (!x_bf16 || !w_bf16 || !topk_idx || !topk_gate) return fail(ctx, MOE_ERR_INVALID_ARG, "null tensor pointer");
   if (num_tokens < 1 || num_tokens > ctx->cfg.max_tokens)
     return fail(ctx, MOE_ERR_INVALID_ARG, "num_tokens %d outside [1, %d]", num_tokens, ctx->cfg.max_tokens);
+  // the dump is written with 16-byte vector stores, the other outputs with 4-byte stores
+  if (reinterpret_cast<uintptr_t>(logits_out) & 15)
+    return fail(ctx, MOE_ERR_INVALID_ARG, "logits_out must be 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(topk_idx) & 3) || (reinterpret_cast<uintptr_t>(topk_gate) & 3) ||
+      (reinterpret_cast<uintptr_t>(alpha_out) & 3))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "topk_idx, topk_gate and alpha_out must be 4-byte aligned");
   if (ctx->cfg.controller == MOE_CTRL_QUANTILE && (!logits_out || !alpha_out))
     return fail(ctx, MOE_ERR_INVALID_ARG, "the quantile controller needs logits_out and alpha_out");
   if (ctx->cfg.controller == MOE_CTRL_QUANTILE && ctx->qb_logits != nullptr) {
@@ -426,6 +433,7 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "controller_kernel launch");
   ctx->launches += 1;
+  ctx->ctrl_steps += 1;
   return MOE_OK;
 }
 
@@ -535,6 +543,13 @@ int moe_loads_peek(moe_route_ctx* ctx, int32_t* loads, void* cuda_stream) {
   return copy_out(ctx, loads, ctx->lay.loads_acc, (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4, st);
 }
 
+int moe_loads_buffer(moe_route_ctx* ctx, int32_t** dev_loads) {
+  if (!ctx || !dev_loads) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  *dev_loads = at<int32_t>(ctx, ctx->lay.loads_acc);
+  return MOE_OK;
+}
+
 int moe_loads_add(moe_route_ctx* ctx, const int32_t* loads, void* cuda_stream) {
   if (!ctx || !loads) return MOE_ERR_INVALID_ARG;
   ctx->err[0] = 0;
@@ -548,9 +563,10 @@ int moe_loads_add(moe_route_ctx* ctx, const int32_t* loads, void* cuda_stream) {
   return MOE_OK;
 }
 
-int moe_state_export(moe_route_ctx* ctx, float* bias, float* e_prev, void* cuda_stream) {
+int moe_state_export(moe_route_ctx* ctx, float* bias, float* e_prev, int64_t* step_host, void* cuda_stream) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   ctx->err[0] = 0;
+  if (step_host) *step_host = ctx->ctrl_steps;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   ctx->last_stream = st;
   const size_t LE = (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4;
@@ -559,9 +575,11 @@ int moe_state_export(moe_route_ctx* ctx, float* bias, float* e_prev, void* cuda_
   return rc;
 }
 
-int moe_state_import(moe_route_ctx* ctx, const float* bias, const float* e_prev, void* cuda_stream) {
+int moe_state_import(moe_route_ctx* ctx, const float* bias, const float* e_prev, int64_t step, void* cuda_stream) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   ctx->err[0] = 0;
+  if (step < -1) return fail(ctx, MOE_ERR_INVALID_ARG, "step must be >= 0 (or -1 to keep the counter)");
+  if (step >= 0) ctx->ctrl_steps = step;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   ctx->last_stream = st;
   const size_t LE = (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4;
@@ -580,8 +598,13 @@ int moe_route_poll(moe_route_ctx* ctx) {
   if (e != cudaSuccess) return cuda_fail(ctx, e, "status read");
   if (st[0] != MOE_OK) {
     cudaMemset(status_ptr(ctx), 0, sizeof st);
-    if (st[0] == MOE_ERR_TIMEOUT)
-      return fail(ctx, MOE_ERR_TIMEOUT, "a bounded device-side wait expired (wait id %d)", st[1]);
+    if (st[0] == MOE_ERR_TIMEOUT) {
+      // the step that gave up is void: its outputs are incomplete and whatever it (and earlier microbatches of
+      // the same step) counted is dropped, so a later controller update cannot consume a partial histogram
+      cudaMemset(ctx->ws + ctx->lay.loads_acc, 0, (size_t)ctx->cfg.num_layers * ctx->cfg.num_experts * 4);
+      ctx->qb_logits = nullptr;
+      return fail(ctx, MOE_ERR_TIMEOUT, "a bounded device-side wait expired (wait id %d); load accumulators cleared", st[1]);
+    }
     if (st[0] == MOE_ERR_STATE)
       return fail(ctx, MOE_ERR_STATE, "controller update on a layer with no routed tokens");
     return fail(ctx, st[0], "device status %d", st[0]);
@@ -608,7 +631,11 @@ int moe_debug_score_gap(float* dev_result, void* cuda_stream) {
   if (!dev_result) return MOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(dev_result, 0, sizeof(float), st) != cudaSuccess) return MOE_ERR_CUDA;
-  score_gap_kernel<<<148 * 8, 256, 0, st>>>(reinterpret_cast<unsigned int*>(dev_result));
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return MOE_ERR_CUDA;
+  score_gap_kernel<<<sms * 8, 256, 0, st>>>(reinterpret_cast<unsigned int*>(dev_result));
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

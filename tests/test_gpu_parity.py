@@ -181,10 +181,14 @@ def test_state_export_import_resume_is_bit_identical():
         return r
     full = run(range(8), binding.Router(1, wl.E, wl.K, wl.H, wl.T))
     first = run(range(4), binding.Router(1, wl.E, wl.K, wl.H, wl.T))
-    b, ep = first.state_export()
+    b, ep, step = first.state_export(with_step=True)
+    assert step == 4                                   # controller updates enqueued so far
     second = binding.Router(1, wl.E, wl.K, wl.H, wl.T)
-    second.state_import(b, ep)
+    second.state_import(b, ep, step=step)
     run(range(4, 8), second)
+    assert second.state_export(with_step=True)[2] == full.state_export(with_step=True)[2] == 8
+    first.state_import(b)                              # step = -1 keeps the context's own counter
+    assert first.state_export(with_step=True)[2] == 4
     for u, v in zip(full.state_export(), second.state_export()):
         np.testing.assert_array_equal(bits(np_(u)), bits(np_(v)))
     for u, v in zip(full.load_stats(), second.load_stats()):
@@ -192,7 +196,7 @@ def test_state_export_import_resume_is_bit_identical():
 
 
 # ------------------------------------------------------------- closed loops
-def _closed_loop(wl, kind, steps, check_rows=None, **kw):
+def _closed_loop(wl, kind, steps, check_rows=None, step_ids=None, **kw):
     """Teacher-forced loop: the GPU runs route + update each step; the oracle
     replays every controller step from the GPU's loads (bitwise) and checks
     the routing of every step against the binary32 chain."""
@@ -206,17 +210,18 @@ def _closed_loop(wl, kind, steps, check_rows=None, **kw):
     alpha = torch.empty(wl.L, wl.T, device=dev)
     differing = checked = 0
     hist = []
-    for t in range(steps):
+    for n_step, t in enumerate(range(steps) if step_ids is None else step_ids):
         x = torch.stack([synth.hidden_states(wl, l, t, dev) for l in range(wl.L)])
         idx, gate = r.route_step(x, w, logits_out=logits, alpha_out=alpha)
         r.controller_update()
         r.poll()
         loads, bias, mxv, mnv = [np_(v) for v in r.load_stats()]
+        gates_gpu = np_(r.gate_stats())
         lg, ix, gt, al = np_(logits), np_(idx), np_(gate), np_(alpha)
         for l in range(wl.L):
             oi = check_exact(lg[l], b[l], wl.K, ix[l], gt[l], al[l])
             np.testing.assert_array_equal(loads[l], np.bincount(oi.ravel(), minlength=wl.E))
-            if check_rows is not None and t % 5 == 0:
+            if check_rows is not None and n_step % 5 == 0:
                 d, c = check_definition(synth.bf16_bits(x[l]), synth.bf16_bits(w[l]), b[l], wl.K, lg[l], ix[l], gt[l],
                                         rows=check_rows)
                 differing += d
@@ -226,8 +231,9 @@ def _closed_loop(wl, kind, steps, check_rows=None, **kw):
                 kind, b[l], ep[l], loads[l], dict(ki=kw.get("ki", 6e-3), kd=kw.get("kd", 6e-3), eta=kw.get("eta", 1e-3), rho=kw.get("qb_ema_rho", 0.0)),
                 center, Q)
             assert bits(mxv[l:l + 1])[0] == bits(np.array([mx]))[0]
+            assert gates_gpu[l] == g                   # open derivative gates (Eq. 11) counted like the oracle
         np.testing.assert_array_equal(bits(bias), bits(b))
-        hist.append((float(mxv.max()), float(mnv.max())))
+        hist.append((float(mxv.max()), float(mnv.max()), int(gates_gpu.sum())))
     if checked:
         assert differing <= max(1, NEAR_TIE_BUDGET * checked)
     return hist
@@ -237,6 +243,7 @@ def test_closed_loop_tiny_top3_id():
     # config "Tiny Top-3-of-768": 20 controller steps, fresh batch per step
     wl = synth.WORKLOADS["tiny_top3"]
     hist = _closed_loop(wl, "id", 20, check_rows=np.arange(0, wl.T, 4))
+    assert max(h[2] for h in hist) > 0                 # the derivative gate opened on routed data at some step
     assert hist[-1][0] < hist[0][0]                    # the controller reduces the overload it started with
 
 
@@ -245,7 +252,7 @@ def test_closed_loop_three_controllers_reduced(kind, K):
     # the Top-3 / Top-5 single-layer comparison at a reduced token count
     wl = synth.WORKLOADS["top3_single"].with_(T=2048, H=512, K=K)
     hist = _closed_loop(wl, kind, 6)
-    assert all(0 <= mx <= wl.E / K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn in hist)
+    assert all(0 <= mx <= wl.E / K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn, _ in hist)
 
 
 @pytest.mark.parametrize("rho", [0.5, 0.9])
@@ -253,14 +260,35 @@ def test_closed_loop_quantile_with_ema(rho):
     # Quantile Balancing with the exponential moving average of Section 3: b = rho b + (1 - rho) Q, bit for bit
     wl = synth.WORKLOADS["top3_single"].with_(T=1024, H=256, K=3)
     hist = _closed_loop(wl, "quantile", 5, qb_ema_rho=rho)
-    assert all(0 <= mx <= wl.E / wl.K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn in hist)
+    assert all(0 <= mx <= wl.E / wl.K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn, _ in hist)
 
 
 def test_closed_loop_quantile_two_layers():
     # Eq. 7 per layer: every layer gets its own target from its own slice of the dump
     wl = synth.WORKLOADS["top3_single"].with_(T=1024, H=256, K=5, L=2)
     hist = _closed_loop(wl, "quantile", 4)
-    assert all(0 <= mx <= wl.E / wl.K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn in hist)
+    assert all(0 <= mx <= wl.E / wl.K - 1 + 1e-4 and 0 <= mn <= 1 for mx, mn, _ in hist)
+
+
+@pytest.mark.parametrize("K", [3, 5])
+def test_quantile_controller_at_full_single_layer_size(K):
+    # the Top-3 / Top-5 single-layer configuration at its own size (T = 16384, H = 2048): one Quantile Balancing
+    # update, target and bias bit-exact against the oracle's sort-based quantile (Eq. 6-7)
+    wl = synth.WORKLOADS["top3_single"].with_(K=K)
+    hist = _closed_loop(wl, "quantile", 1)
+    assert 0 <= hist[0][0] <= wl.E / K - 1 + 1e-4
+
+
+def test_closed_loop_drifting_deep_stack_opens_the_derivative_gate():
+    # deep-stack configuration at a reduced token count: the cluster means drift linearly over the 500 steps of
+    # the workload, so consecutive controller steps taken from steps spread over the drift see the imbalance of
+    # some experts grow -- the derivative gate of Algorithm 1 line 9 opens on routed data, and the number of
+    # open gates per layer equals the oracle's
+    wl = synth.WORKLOADS["top10_deep"].with_(L=6, T=2048)
+    ids = [0, 40, 90, 150, 220, 300, 380, 450, 499]
+    hist = _closed_loop(wl, "id", len(ids), step_ids=ids)
+    assert hist[0][2] == 0                       # first step: previous error is zero, every gate closed
+    assert max(h[2] for h in hist[1:]) > 0       # later steps: gates open somewhere
 
 
 def test_quantile_target_count_property_on_gpu_result():
@@ -311,6 +339,20 @@ def test_argument_errors_are_reported_not_raised_by_cuda():
     rq = binding.Router(1, 768, 3, 64, 128, controller="quantile")
     with pytest.raises(binding.MoeRouteError):
         rq.route_step(x[:, :128].contiguous(), w)        # quantile controller without the dump buffers
+    # misaligned output buffers are refused on the host (the dump is written with 16-byte stores)
+    x1 = x[:, :128].contiguous()
+    n0 = r.launch_count()
+    buf = torch.empty(128 * 768 + 8, device="cuda")
+    for off in (1, 2, 3):
+        with pytest.raises(binding.MoeRouteError) as ei:
+            r.route_step(x1, w, logits_out=buf[off:off + 128 * 768])
+        assert ei.value.code == binding.MOE_ERR_INVALID_ARG
+    raw = torch.empty(128 * 10 * 4 + 8, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.MoeRouteError) as ei:
+        r.route_step(x1, w, topk_idx=raw[2:2 + 128 * 10 * 4].view(torch.int32))
+    assert ei.value.code == binding.MOE_ERR_INVALID_ARG
+    assert r.launch_count() == n0                        # nothing was launched
+    r.route_step(x1, w, logits_out=buf[4:4 + 128 * 768])  # 16-byte aligned offset is fine
     assert r.poll(raise_on_error=False) == binding.MOE_OK
 
 
@@ -476,6 +518,51 @@ def test_bounded_wait_gives_up_and_reports_timeout():
     np.testing.assert_array_equal(np_(r.loads_peek()), 2 * res["loads"])
 
 
+def test_routing_kernel_gives_up_cleanly_when_its_waits_run_out():
+    # a context whose device-side waits are bounded to a single retry: the first wait for a tile that is still
+    # in flight runs out, every role of every CTA leaves its loop, copies and MMAs in flight drain, tensor memory
+    # is released and the kernel returns; the host sees MOE_ERR_TIMEOUT, the void step's counts are dropped, and
+    # the device keeps working (a context with the default bound routes the same batch correctly afterwards)
+    T, H, E, K = 256, 64, 768, 10
+    good = route_once(T, H, E, K, seed=11)
+    r = binding.Router(1, E, K, H, T, spin_limit=1)
+    r.route_step(good["x"], good["w"])
+    assert r.poll(raise_on_error=False) == binding.MOE_ERR_TIMEOUT
+    assert not np_(r.loads_peek()).any()                         # partial histogram dropped
+    assert r.poll(raise_on_error=False) == binding.MOE_OK        # sticky status cleared
+    bias, e_prev = [np_(v) for v in r.state_export()]
+    assert not bias.any() and not e_prev.any()                   # controller state untouched
+    again = route_once(T, H, E, K, seed=11)
+    np.testing.assert_array_equal(again["idx"], good["idx"])
+    np.testing.assert_array_equal(again["loads"], good["loads"])
+    full_check(again, K)
+
+
+@pytest.mark.parametrize("name,L,T", [("top10_deep", 48, 700), ("top10_large", 60, 700)])
+def test_all_layers_of_the_deep_configurations_in_one_launch(name, L, T):
+    # every layer of the 48- and 60-layer configurations in ONE routing call, at their own hidden size and a
+    # reduced, ragged token count (three tile pairs per layer: 144 / 180 work items walked by the persistent
+    # grid across layer changes): all tokens of all layers against the binary32 chain, per-layer loads, and a
+    # row sample against the fp64 definition
+    wl = synth.WORKLOADS[name].with_(T=T)
+    assert wl.L == L
+    dev = "cuda"
+    g = torch.Generator().manual_seed(L)
+    bias = torch.randn(L, wl.E, generator=g) * 0.01
+    x = torch.stack([synth.hidden_states(wl, l, 1, dev) for l in range(L)])
+    w = torch.stack([synth.router_weights(wl, l, dev) for l in range(L)])
+    res = route_once(T, wl.H, wl.E, wl.K, L=L, bias=bias, want_alpha=True, x=x, w=w)
+    full_check(res, wl.K, rows=np.arange(3, T, 16))
+    # the same call without the dump (the timed configuration) gives the same selections
+    r = binding.Router(L, wl.E, wl.K, wl.H, T)
+    r.state_import(bias=bias.cuda().contiguous())
+    idx, gate = r.route_step(x, w)
+    r.poll()
+    np.testing.assert_array_equal(np_(idx), res["idx"])
+    np.testing.assert_array_equal(bits(np_(gate)), bits(res["gate"]))
+    np.testing.assert_array_equal(np_(r.loads_peek()), res["loads"])
+
+
 # ------------------------------------------------ full-size configurations
 def _full_size(wl, layers, steps=1, sample=192):
     """Full T and H of a configuration (a few layers of it), in the launch
@@ -532,4 +619,4 @@ def test_full_size_deep_stack_layers():
 
 
 def test_full_size_large_scale_layers():
-    _full_size(synth.WORKLOADS["top10_large"], layers=2, sample=64)
+    _full_size(synth.WORKLOADS["top10_large"], layers=2, sample=256)
