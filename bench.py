@@ -523,6 +523,9 @@ def main():
     repeats = max(1, math.ceil(args.min_region_s * 1e3 / max(1e-6, est_ms * args.steps)))
     sampler.start()
     total_ms, route_ms, launches = job.timed(args.steps, repeats)
+    while total_ms < args.min_region_s * 1e3:          # the estimate was too high: time a longer region
+        repeats = max(repeats + 1, math.ceil(1.1 * repeats * args.min_region_s * 1e3 / total_ms))
+        total_ms, route_ms, launches = job.timed(args.steps, repeats)
     clocks = sampler.stop()
     loads, bias, maxvio, minvio = job.router.load_stats()
     gate_open = int(job.router.gate_stats().sum())
@@ -558,6 +561,9 @@ def main():
             o_steps = max(3, args.steps)
             o_rep = max(1, math.ceil(args.min_region_s * 1e3 / max(1e-6, o_est * o_steps)))
             o_ms, o_route, _ = oj.timed(o_steps, o_rep)
+            while o_ms < args.min_region_s * 1e3:
+                o_rep = max(o_rep + 1, math.ceil(1.1 * o_rep * args.min_region_s * 1e3 / o_ms))
+                o_ms, o_route, _ = oj.timed(o_steps, o_rep)
             oj.router.poll()
             if dist is not None:
                 t = torch.tensor([o_ms], device=dev, dtype=torch.float64)

@@ -349,7 +349,7 @@ def test_argument_errors_are_reported_not_raised_by_cuda():
         assert ei.value.code == binding.MOE_ERR_INVALID_ARG
     raw = torch.empty(128 * 10 * 4 + 8, dtype=torch.uint8, device="cuda")
     with pytest.raises(binding.MoeRouteError) as ei:
-        r.route_step(x1, w, topk_idx=raw[2:2 + 128 * 10 * 4].view(torch.int32))
+        r.route_step(x1, w, topk_idx=raw[2:2 + 128 * 10 * 4])      # byte tensor: only its address is used
     assert ei.value.code == binding.MOE_ERR_INVALID_ARG
     assert r.launch_count() == n0                        # nothing was launched
     r.route_step(x1, w, logits_out=buf[4:4 + 128 * 768])  # 16-byte aligned offset is fine
@@ -512,10 +512,11 @@ def test_bounded_wait_gives_up_and_reports_timeout():
     r.debug_wait_timeout(spin_limit=2000)
     assert r.poll(raise_on_error=False) == binding.MOE_ERR_TIMEOUT
     assert r.poll(raise_on_error=False) == binding.MOE_OK          # sticky status cleared by the poll
+    assert not np_(r.loads_peek()).any()                           # a timed-out iteration is void: counts dropped
     idx, gate = r.route_step(res["x"], res["w"])
     r.poll()
     np.testing.assert_array_equal(np_(idx), res["idx"])
-    np.testing.assert_array_equal(np_(r.loads_peek()), 2 * res["loads"])
+    np.testing.assert_array_equal(np_(r.loads_peek()), res["loads"])
 
 
 def test_routing_kernel_gives_up_cleanly_when_its_waits_run_out():
