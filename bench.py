@@ -84,7 +84,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) every few ms."""
 
     def __init__(self, index):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.power, self.reasons, self.max_mhz = [], [], set(), None
         self._stop = threading.Event()
         self._th = None
         try:
@@ -103,6 +103,7 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
                 mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
                 for k, bit in names.items():
                     if mask & bit:
@@ -123,7 +124,8 @@ class ClockSampler:
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
         return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w": statistics.median(self.power) if self.power else None}
 
 
 def cpu_oracle_rate(wl, threads, tokens_per_thread, keep=False):
@@ -258,6 +260,8 @@ def run_aux(args, wl):
 class Job:
     """Inputs, outputs and context of one workload on one rank."""
 
+    chunk_split = 0      # moe_route_config.chunk_split of every context made here (0 = the library chooses)
+
     def __init__(self, wl, dev, rank, world, dist):
         from paper_2609_39137_b200 import binding, dp
         self.wl, self.dev, self.dist, self.dp = wl, dev, dist, dp
@@ -272,7 +276,8 @@ class Job:
             self.xs.append(x)
         self.idx = torch.empty(wl.L, wl.T, wl.K, dtype=torch.int32, device=dev)
         self.gate = torch.empty(wl.L, wl.T, wl.K, dtype=torch.float32, device=dev)
-        self.router = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T, controller="id", device=dev)
+        self.router = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T, controller="id", device=dev,
+                                     chunk_split=Job.chunk_split)
 
     def step(self, i):
         self.router.route_step(self.xs[i % self.ring], self.w, self.idx, self.gate)
@@ -476,6 +481,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-configs", action="store_true", help="time only the chosen workload")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--chunk-split", type=int, default=0, choices=[0, 1, 2],
+                    help="scheduling of the expert chunks (moe_route_config.chunk_split); 0 = the library chooses")
     ap.add_argument("--aux", action="store_true", help="time the calls outside the step (one GPU) and exit")
     args = ap.parse_args()
 
@@ -516,6 +523,7 @@ def main():
 
     pk = peaks()
     sampler = ClockSampler(local_rank)
+    Job.chunk_split = args.chunk_split
 
     # ---- headline workload
     job = Job(wl, dev, rank, world, dist)

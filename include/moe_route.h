@@ -88,6 +88,12 @@ typedef struct {
                            0 = [L][E][H] (W_r in R^{E x d} as Section 2.2 writes it, hidden contiguous),
                            1 = [L][H][E] (expert contiguous); the library then transposes into
                            L*E*H*2 bytes of workspace before every routing launch */
+  int32_t chunk_split;  /* scheduling of the 256-expert chunks of a token tile (E > 256 only; results are
+                           identical either way): 1 = one CTA pair walks all chunks of its tile and finishes the
+                           rows in its epilogue; 2 = the chunks of a tile go to different CTA pairs that run at
+                           the same time (the tile is streamed from HBM once) and a merge kernel finishes the
+                           rows from L*ceil(E/256)*max_tokens*(K+1)*8 bytes of workspace; 0 = chosen by the
+                           hidden size (2 when the tiles of all resident pairs no longer fit in L2) */
 } moe_route_config;
 
 /* Fills *cfg with the paper's defaults (Ki = Kd = 6e-3, eta = 1e-3, rho = 0,
@@ -262,6 +268,15 @@ int moe_quantile_target_static(const float* logits, const float* alpha, int32_t 
  * gives up, the kernel returns normally, and the next moe_route_poll reports
  * MOE_ERR_TIMEOUT (wait id 99); the context stays usable. */
 int moe_debug_wait_timeout(moe_route_ctx* ctx, int32_t spin_limit, void* cuda_stream);
+
+/* Validation utility for the give-up path of the routing kernel itself: in the
+ * NEXT moe_route_step of this context (only that one) every producer warp stops
+ * issuing loads after `after_loads` (>= 1) pipeline stages, as if the copies had
+ * stalled.  Nothing is left in flight; the consumers' bounded waits run out (use
+ * a context with a small spin_limit so that this takes milliseconds), every role
+ * of every CTA leaves its loop, tensor memory is released, the kernel returns,
+ * and moe_route_poll reports MOE_ERR_TIMEOUT.  Host call; nothing is enqueued. */
+int moe_debug_route_stall(moe_route_ctx* ctx, int32_t after_loads);
 
 /* Number of kernels this context has launched so far. */
 int64_t moe_route_launch_count(const moe_route_ctx* ctx);

@@ -24,7 +24,7 @@ SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_i
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_loads_buffer", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
            "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static",
-           "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout", "moe_score_stats"]
+           "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout", "moe_score_stats", "moe_debug_route_stall"]
 
 
 class MoeRouteConfig(C.Structure):
@@ -32,7 +32,7 @@ class MoeRouteConfig(C.Structure):
                 ("top_k", C.c_int32), ("hidden", C.c_int32), ("max_tokens", C.c_int32), ("controller", C.c_int32),
                 ("ki", C.c_float), ("kd", C.c_float), ("eta", C.c_float), ("qb_ema_rho", C.c_float),
                 ("center", C.c_int32), ("spin_limit", C.c_int32), ("host_staging", C.c_int32),
-                ("w_layout", C.c_int32)]
+                ("w_layout", C.c_int32), ("chunk_split", C.c_int32)]
 
 
 class MoeRouteError(RuntimeError):
@@ -79,6 +79,7 @@ def load():
     L.moe_route_destroy.argtypes = [vp]
     L.moe_debug_score_gap.argtypes = [vp, vp]
     L.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
+    L.moe_debug_route_stall.argtypes = [vp, i32]
     L.moe_score_stats.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.moe_quantile_target_static.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     _lib = L
@@ -127,7 +128,7 @@ class Router:
 
     def __init__(self, num_layers, num_experts, top_k, hidden, max_tokens, controller="id", ki=None, kd=None,
                  eta=None, qb_ema_rho=None, center=None, spin_limit=0, host_staging=False, w_layout=0,
-                 device="cuda"):
+                 chunk_split=0, device="cuda"):
         self.lib = load()
         cfg = default_config(num_layers, num_experts, top_k, hidden, max_tokens)
         cfg.controller = CONTROLLERS[controller] if isinstance(controller, str) else int(controller)
@@ -139,6 +140,7 @@ class Router:
         cfg.spin_limit = spin_limit
         cfg.host_staging = int(bool(host_staging))
         cfg.w_layout = int(w_layout)
+        cfg.chunk_split = int(chunk_split)
         self.cfg = cfg
         self.L, self.E, self.K, self.H, self.max_tokens = num_layers, num_experts, top_k, hidden, max_tokens
         self.device = torch.device(device)
@@ -269,6 +271,10 @@ class Router:
     def debug_wait_timeout(self, spin_limit=2000):
         """Launches the bounded-wait probe (a wait nothing satisfies); poll() then reports MOE_ERR_TIMEOUT."""
         self._check(self.lib.moe_debug_wait_timeout(self.h, spin_limit, _stream()))
+
+    def debug_route_stall(self, after_loads=2):
+        """The next route_step's producers stop after `after_loads` pipeline stages (validation of the give-up path)."""
+        self._check(self.lib.moe_debug_route_stall(self.h, int(after_loads)))
 
     def launch_count(self):
         return int(self.lib.moe_route_launch_count(self.h))

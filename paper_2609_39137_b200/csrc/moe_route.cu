@@ -16,6 +16,7 @@
 #include "quantile_kernel.cuh"
 #include "score_stats_kernel.cuh"
 #include "route_kernel.cuh"
+#include "route_merge_kernel.cuh"
 
 namespace {
 
@@ -31,8 +32,20 @@ struct Layout {
   size_t stat_P, stat_H, stat_aux, ent_part;   // per-CTA partial sums of moe_score_stats (written before they are read)
   size_t stage_x, stage_w, stage_idx, stage_gate;
   size_t w_t;   // [L][E][H] bf16 copy of the weights when they are given as [L][H][E]
+  size_t cand;  // [L][chunks][max_tokens][K+1] (score, expert) pairs, chunk-split scheduling only
   size_t total;
 };
+
+// Chunk-split scheduling (the expert chunks of a token tile go to different CTA pairs, a merge kernel
+// finishes): chosen when one CTA pair re-reading its tile once per chunk would push the tiles of all
+// resident pairs out of L2 -- 74 pairs x 256 tokens x hidden x 2 bytes exceeds the 126 MB L2 beyond
+// hidden ~ 3300 -- and there is more than one chunk.
+bool use_chunk_split(const moe_route_config& c) {
+  if (c.num_experts <= kBN) return false;
+  if (c.chunk_split == 1) return false;
+  if (c.chunk_split == 2) return true;
+  return c.hidden > 3072;
+}
 
 Layout make_layout(const moe_route_config& c) {
   Layout l{};
@@ -71,6 +84,10 @@ Layout make_layout(const moe_route_config& c) {
     l.stage_gate = take(LT * c.top_k * 4);
   }
   if (c.w_layout == 1) l.w_t = take(LE * c.hidden * 2);
+  if (use_chunk_split(c)) {
+    const size_t chunks = (size_t)(c.num_experts + kBN - 1) / kBN;
+    l.cand = take((size_t)c.num_layers * chunks * c.max_tokens * (c.top_k + 1) * sizeof(float2));
+  }
   l.total = o;
   return l;
 }
@@ -88,6 +105,7 @@ bool config_ok(const moe_route_config* c) {
   if (c->center < -1 || c->center > 1) return false;
   if (c->spin_limit < 0) return false;
   if (c->w_layout != 0 && c->w_layout != 1) return false;
+  if (c->chunk_split < 0 || c->chunk_split > 2) return false;
   return true;
 }
 
@@ -118,6 +136,7 @@ struct moe_route_ctx {
   cudaStream_t last_stream;
   int64_t launches;
   int64_t ctrl_steps;   // controller updates enqueued so far (exported / restored with the controller state)
+  int stall_next;       // moe_debug_route_stall: applies to the next routing launch only
   // cached TMA descriptors
   const void* map_x_ptr;
   const void* map_w_ptr;
@@ -233,15 +252,44 @@ int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, in
   rp.topk_idx = idx; rp.topk_gate = gate; rp.logits_out = logits; rp.alpha_out = alpha;
   rp.status = status_ptr(ctx);
   rp.spin_limit = c.spin_limit > 0 ? (uint32_t)c.spin_limit : 0x7fffffffu;
+  const int need = c.top_k + (alpha ? 1 : 0);
+  rp.stall_after = ctx->stall_next;
+  ctx->stall_next = 0;
+  rp.split = use_chunk_split(c) ? 1 : 0;
+  if (rp.split) {
+    rp.num_items *= rp.num_chunks;
+    rp.cand_len = need;
+    rp.cand = at<float2>(ctx, ctx->lay.cand);
+  }
   const int max_pairs = ctx->num_sms / 2;
   const int grid = 2 * (rp.num_items < max_pairs ? rp.num_items : max_pairs);   // clusters of 2 CTAs
-  const int need = c.top_k + (alpha ? 1 : 0);
-  if (need <= 3) return launch_route<3>(ctx, rp, grid, st);
-  if (need <= 5) return launch_route<5>(ctx, rp, grid, st);
-  if (need <= 8) return launch_route<8>(ctx, rp, grid, st);
-  if (need <= 10) return launch_route<10>(ctx, rp, grid, st);
-  if (need <= 11) return launch_route<11>(ctx, rp, grid, st);   // Top-10 with the alpha output (quantile controller)
-  return launch_route<17>(ctx, rp, grid, st);
+  int rc;
+  if (need <= 3) rc = launch_route<3>(ctx, rp, grid, st);
+  else if (need <= 5) rc = launch_route<5>(ctx, rp, grid, st);
+  else if (need <= 8) rc = launch_route<8>(ctx, rp, grid, st);
+  else if (need <= 10) rc = launch_route<10>(ctx, rp, grid, st);
+  else if (need <= 11) rc = launch_route<11>(ctx, rp, grid, st);   // Top-10 with the alpha output (quantile controller)
+  else rc = launch_route<17>(ctx, rp, grid, st);
+  if (rc != MOE_OK || !rp.split) return rc;
+  // chunk-split scheduling: merge the chunks' candidate lists into indices, gates, alpha and loads
+  MergeParams mp{};
+  mp.T = T; mp.E = c.num_experts; mp.K = c.top_k; mp.num_chunks = rp.num_chunks; mp.cand_len = need;
+  mp.cand = rp.cand; mp.bias = rp.bias; mp.loads = rp.loads;
+  mp.topk_idx = idx; mp.topk_gate = gate; mp.alpha_out = alpha;
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3((T + kMergeRowsPerCta - 1) / kMergeRowsPerCta, c.num_layers);
+  lc.blockDim = dim3(kMergeThreads);
+  lc.dynamicSmemBytes = 0;
+  lc.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &attr;
+  lc.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&lc, route_merge_kernel, mp);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "route_merge_kernel launch");
+  ctx->launches += 1;
+  return MOE_OK;
 }
 
 }  // namespace
@@ -267,6 +315,7 @@ void moe_route_default_config(moe_route_config* cfg, int32_t num_layers, int32_t
   cfg->spin_limit = 0;
   cfg->host_staging = 0;
   cfg->w_layout = 0;
+  cfg->chunk_split = 0;
 }
 
 size_t moe_route_workspace_bytes(const moe_route_config* cfg) {
@@ -683,6 +732,13 @@ int moe_debug_wait_timeout(moe_route_ctx* ctx, int32_t spin_limit, void* cuda_st
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "wait_timeout_probe_kernel launch");
   ctx->launches += 1;
+  return MOE_OK;
+}
+
+int moe_debug_route_stall(moe_route_ctx* ctx, int32_t after_loads) {
+  if (!ctx || after_loads < 1) return MOE_ERR_INVALID_ARG;
+  ctx->err[0] = 0;
+  ctx->stall_next = after_loads;
   return MOE_OK;
 }
 

@@ -46,6 +46,45 @@ def test_route_edge_shapes(T, H, E, K):
     full_check(res, K)
 
 
+@pytest.mark.parametrize("T,H,E,K,L,alpha", [
+    (128, 64, 768, 3, 1, False),      # one tile pair, three chunk items
+    (300, 512, 768, 10, 1, True),     # ragged tail, alpha from the merged lists
+    (1000, 256, 768, 5, 3, True),     # layers
+    (513, 192, 1000, 16, 2, False),   # four chunks, the last one mostly padding; generic (insertion) selection
+    (130, 64, 1000, 15, 1, True),
+    (700, 320, 264, 8, 2, True),      # second chunk holds 8 experts: fewer than K + 1 per chunk list
+    (2100, 128, 512, 1, 1, True),     # more rows than one merge CTA takes
+])
+def test_chunk_split_scheduling_matches_oracle_and_fused_path(T, H, E, K, L, alpha):
+    # the expert chunks of a tile routed by different CTA pairs and merged by the second kernel: parity with the
+    # oracle, and bit-identical to the schedule that finishes the rows in the routing kernel's epilogue
+    g = torch.Generator().manual_seed(T + K)
+    bias = torch.randn(L, E, generator=g) * 0.02
+    res = route_once(T, H, E, K, L, bias=bias, seed=T, want_alpha=alpha, chunk_split=2)
+    full_check(res, K)
+    fused = route_once(T, H, E, K, L, bias=bias, seed=T, want_alpha=alpha, chunk_split=1)
+    for k in ("logits", "idx", "gate", "loads") + (("alpha",) if alpha else ()):
+        np.testing.assert_array_equal(bits(res[k]) if res[k].dtype == np.float32 else res[k],
+                                      bits(fused[k]) if fused[k].dtype == np.float32 else fused[k])
+    assert res["r"].launch_count() == fused["r"].launch_count() + 1      # the merge kernel
+
+
+def test_chunk_split_exact_ties_across_chunks_pick_lowest_index():
+    # every score equal: the winners are the K lowest indices, all in the first chunk; with a bias plateau that
+    # spans chunk boundaries the merge has to break ties between lists by expert index
+    T, H, E, K = 200, 64, 768, 10
+    x = torch.zeros(1, T, H, device="cuda", dtype=torch.bfloat16)
+    res = route_once(T, H, E, K, x=x, chunk_split=2)
+    assert np.all(res["idx"][0] == np.arange(K)[None, :])
+    bias = torch.zeros(1, E)
+    bias[0, 250:260] = 0.25           # straddles chunks 0 and 1
+    bias[0, 600:604] = 0.25           # chunk 2
+    res = route_once(T, H, E, K, x=x, bias=bias, want_alpha=True, chunk_split=2)
+    assert np.all(res["idx"][0] == np.arange(250, 260)[None, :])
+    assert np.all(res["alpha"][0] == np.float32(0.75))
+    full_check(res, K)
+
+
 def test_route_operand_layout_one_hot():
     # one-hot router rows: logit[t][e] = x[t][h(e)] exactly -- exposes any
     # swizzle / descriptor / transposition error
@@ -440,7 +479,7 @@ def test_route_random_shapes_bit_exact(seed):
     if quantise:
         x, w, bias = torch.round(x), torch.round(w * 4) / 4, torch.round(bias * 8) / 8
     res = route_once(T, H, E, K, L=L, bias=bias, want_alpha=(K < 16), x=x.cuda().to(torch.bfloat16),
-                     w=w.cuda().to(torch.bfloat16))
+                     w=w.cuda().to(torch.bfloat16), chunk_split=1 + seed % 2)
     for l in range(L):
         a = None if res["alpha"] is None else res["alpha"][l]
         oi = check_exact(res["logits"][l], res["bias"][l], K, res["idx"][l], res["gate"][l], a)
@@ -519,24 +558,29 @@ def test_bounded_wait_gives_up_and_reports_timeout():
     np.testing.assert_array_equal(np_(r.loads_peek()), res["loads"])
 
 
-def test_routing_kernel_gives_up_cleanly_when_its_waits_run_out():
-    # a context whose device-side waits are bounded to a single retry: the first wait for a tile that is still
-    # in flight runs out, every role of every CTA leaves its loop, copies and MMAs in flight drain, tensor memory
-    # is released and the kernel returns; the host sees MOE_ERR_TIMEOUT, the void step's counts are dropped, and
-    # the device keeps working (a context with the default bound routes the same batch correctly afterwards)
-    T, H, E, K = 256, 64, 768, 10
-    good = route_once(T, H, E, K, seed=11)
-    r = binding.Router(1, E, K, H, T, spin_limit=1)
+@pytest.mark.parametrize("chunk_split,after", [(1, 2), (2, 3)])
+def test_routing_kernel_gives_up_cleanly_when_its_waits_run_out(chunk_split, after):
+    # the producers of ONE routing launch stop issuing loads after a few pipeline stages (nothing is left in
+    # flight, no fault, no endless loop): the MMA warp's bounded wait for the next stage runs out, every role of
+    # every CTA leaves its loop, tensor memory is released and the kernel returns; the host sees
+    # MOE_ERR_TIMEOUT, the void step's counts are dropped, the controller state is untouched, and the same
+    # context routes the same batch correctly afterwards
+    T, H, E, K, L = 700, 256, 768, 10, 2
+    good = route_once(T, H, E, K, L=L, seed=11, chunk_split=chunk_split)
+    r = binding.Router(L, E, K, H, T, spin_limit=4000, chunk_split=chunk_split)
+    r.debug_route_stall(after_loads=after)
     r.route_step(good["x"], good["w"])
     assert r.poll(raise_on_error=False) == binding.MOE_ERR_TIMEOUT
+    assert "wait" in r.lib.moe_last_error(r.h).decode()
     assert not np_(r.loads_peek()).any()                         # partial histogram dropped
     assert r.poll(raise_on_error=False) == binding.MOE_OK        # sticky status cleared
     bias, e_prev = [np_(v) for v in r.state_export()]
     assert not bias.any() and not e_prev.any()                   # controller state untouched
-    again = route_once(T, H, E, K, seed=11)
-    np.testing.assert_array_equal(again["idx"], good["idx"])
-    np.testing.assert_array_equal(again["loads"], good["loads"])
-    full_check(again, K)
+    idx, gate = r.route_step(good["x"], good["w"])               # the stall applied to one launch only
+    r.poll()
+    np.testing.assert_array_equal(np_(idx), good["idx"])
+    np.testing.assert_array_equal(bits(np_(gate)), bits(good["gate"]))
+    np.testing.assert_array_equal(np_(r.loads_peek()), good["loads"])
 
 
 @pytest.mark.parametrize("name,L,T", [("top10_deep", 48, 700), ("top10_large", 60, 700)])
