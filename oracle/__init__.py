@@ -63,6 +63,7 @@ def lib():
             L.oracle_id_update.argtypes = [_f32p, _f32p, _f32p, _i64, C.c_float, C.c_float, C.c_int, _i32p]
             L.oracle_fixed_step_update.argtypes = [_f32p, _f32p, _f32p, _i64, C.c_float, C.c_int]
             L.oracle_quantile_target.argtypes = [_f32p, _f32p, _i64, _i64, _i64, _f32p]
+            L.oracle_quantile_target_hist.argtypes = [_f32p, _f32p, _i64, _i64, _i64, _i64, C.c_float, _f32p, _i64p]
             L.oracle_quantile_update.argtypes = [_f32p, _f32p, _f32p, _f32p, _i64, C.c_float, C.c_int]
             L.oracle_violations.argtypes = [_i64p, _i64, _f32p, _f32p]
             L.oracle_load_diagnostics.argtypes = [_i64p, _i32p, _f32p, _f32p, _i64, _f32p]
@@ -244,6 +245,21 @@ def quantile_target(z32, alpha, K):
     if lib().oracle_quantile_target(_p(z32, _f32p), _p(alpha, _f32p), m, E, K, _p(Q, _f32p)):
         raise ValueError("oracle_quantile_target failed")
     return Q
+
+
+def quantile_target_hist(z32, alpha, K, bins, value_range, return_hist=False):
+    """Footnote to Eq. 7: Q_j estimated from a per-expert margin histogram (`bins` uniform bins over
+    [-value_range, value_range), linear interpolation inside the bin; this build's reading)."""
+    z32 = _arr(z32, np.float32)
+    alpha = _arr(alpha, np.float32)
+    m, E = z32.shape
+    Q = np.empty(E, np.float32)
+    hist = np.zeros((E, bins), np.int64) if return_hist else None
+    rc = lib().oracle_quantile_target_hist(_p(z32, _f32p), _p(alpha, _f32p), m, E, K, bins, float(value_range),
+                                           _p(Q, _f32p), _p(hist, _i64p) if return_hist else None)
+    if rc:
+        raise ValueError("oracle_quantile_target_hist failed")
+    return (Q, hist) if return_hist else Q
 
 
 def quantile_update(b, e_prev, e, Q, rho=0.0, center=False):

@@ -341,6 +341,65 @@ int oracle_quantile_target(const float *z, const float *alpha, int64_t m,
 }
 
 /*
+ * Quantile Balancing target estimated from a per-expert margin histogram
+ * (footnote to Eq. 7, Section 2.3: "at scale" the quantile is estimated from
+ * such a histogram).  The paper fixes neither bins nor range nor the rule
+ * inside a bin -- PARITY UNPINNED against the paper; the reading taken here:
+ *   B uniform bins over [-range, +range), bin width h = 2*range/B;
+ *   margin d = sigmoid_f32(z_ij) - alpha_i in binary32 (as in the exact form);
+ *   bin k = floor((d + range) * inv_h) with inv_h = (float)B / (2*range), both
+ *   operations rounded to binary32, clamped to [0, B-1] (margins outside the
+ *   range count in the end bins);
+ *   same nearest rank as the exact form, r = m - floor(m*K/E) in [1, m];
+ *   k* = the bin that holds the r-th smallest margin (below = count of the
+ *   bins before it, cnt = its own count); estimate by linear interpolation
+ *   at the middle of the r-th margin's share of the bin, in binary64,
+ *     est = -range + (k* + ((r - below) - 0.5) / cnt) * h,   Q_j = -(float)est.
+ * Since the exact r-th smallest margin lies in bin k* too, |est - exact| < h
+ * whenever that margin is inside the range.  hist (may be NULL) receives the
+ * counts, [E][B].
+ */
+int oracle_quantile_target_hist(const float *z, const float *alpha, int64_t m,
+                                int64_t E, int64_t K, int64_t B, float range,
+                                float *Q, int64_t *hist)
+{
+    if (m < 1 || B < 1 || !(range > 0.0f)) return -1;
+    int64_t *cnt = (int64_t *)malloc((size_t)B * sizeof *cnt);
+    if (!cnt) return -1;
+    int64_t r = m - (m * K) / E;
+    if (r < 1) r = 1;
+    if (r > m) r = m;
+    const float inv_h = (float)B / (2.0f * range);
+    const double h = 2.0 * (double)range / (double)B;
+    for (int64_t j = 0; j < E; ++j) {
+        for (int64_t k = 0; k < B; ++k) cnt[k] = 0;
+        for (int64_t i = 0; i < m; ++i) {
+            float d = oracle_sigmoid_f32(z[i * E + j]) - alpha[i];
+            float shifted = d + range;
+            float u = shifted * inv_h;
+            int64_t k = 0;
+            if (u >= 0.0f) {
+                float fl = floorf(u);
+                k = (fl >= (float)B) ? B - 1 : (int64_t)fl;
+            }
+            cnt[k] += 1;
+        }
+        int64_t below = 0, kstar = 0;
+        for (int64_t k = 0; k < B; ++k) {
+            if (r <= below + cnt[k]) { kstar = k; break; }
+            below += cnt[k];
+        }
+        double inside = ((double)(r - below) - 0.5) / (double)cnt[kstar];
+        double est = -(double)range + ((double)kstar + inside) * h;
+        Q[j] = -(float)est;
+        if (hist)
+            for (int64_t k = 0; k < B; ++k) hist[j * B + k] = cnt[k];
+    }
+    free(cnt);
+    return 0;
+}
+
+/*
  * Quantile Balancing update with the diagnostic EMA of Section 3:
  *   b <- rho * b + (1 - rho) * Q, 0 <= rho < 1; rho = 0 stores Q unchanged.
  * binary32: (rho * b) + ((1 - rho) * Q), no fused multiply-add.

@@ -417,6 +417,59 @@ def test_quantile_target_places_q_tokens_above_cutoff():
     np.testing.assert_allclose(b5, 0.5 * b + 0.5 * Q, atol=1e-8)
 
 
+def test_quantile_histogram_estimate_hand_example():
+    # logits 0 give the score 0.5 exactly, so alpha_i = 0.5 - d_i plants the margins d = -0.5, -0.25, 0.25, 0.5.
+    # B = 4 bins over [-1, 1): edges -1, -0.5, 0, 0.5, 1 -> counts [0, 2, 1, 1].  E = 4, K = 1: r = 4 - 1 = 3,
+    # the third smallest margin (0.25) sits alone in bin 2 (below = 2, count = 1): est = -1 + (2 + 0.5) * 0.5
+    # = 0.25, Q = -0.25.  With K = 2: r = 2, bin 1 (below = 0, count = 2): est = -1 + (1 + 1.5 / 2) * 0.5 = -0.125.
+    d = np.array([-0.5, -0.25, 0.25, 0.5], np.float32)
+    z = np.zeros((4, 4), np.float32)
+    alpha = (np.float32(0.5) - d).astype(np.float32)
+    Q, hist = oracle.quantile_target_hist(z, alpha, 1, 4, 1.0, return_hist=True)
+    np.testing.assert_array_equal(hist, np.tile(np.array([0, 2, 1, 1]), (4, 1)))
+    np.testing.assert_array_equal(Q, np.full(4, -0.25, np.float32))
+    np.testing.assert_array_equal(oracle.quantile_target_hist(z, alpha, 2, 4, 1.0), np.full(4, 0.125, np.float32))
+    # margins outside the range count in the end bins: range 0.375 -> bins of width 0.1875 over [-0.375, 0.375)
+    _, hist = oracle.quantile_target_hist(z, alpha, 1, 4, 0.375, return_hist=True)
+    np.testing.assert_array_equal(hist[0], np.array([2, 0, 0, 2]))
+
+
+@pytest.mark.parametrize("bins,value_range", [(64, 1.0), (1024, 1.0), (4096, 2.0), (512, 0.25)])
+def test_quantile_histogram_estimate_is_within_one_bin_of_the_exact_target(bins, value_range):
+    # the exact r-th smallest margin lies in the bin the estimate interpolates in: |estimate - exact| < bin width
+    # wherever the exact value is inside the range; counts of every expert sum to m; finer bins converge
+    rng = np.random.default_rng(61)
+    m, E, K = 700, 48, 5
+    z = (rng.standard_normal((m, E)) * 1.5).astype(np.float32)
+    b = (rng.standard_normal(E) * 0.05).astype(np.float32)
+    _, _, alpha = oracle.route_f32(z, b, K)
+    exact = oracle.quantile_target(z, alpha, K)
+    est, hist = oracle.quantile_target_hist(z, alpha, K, bins, value_range, return_hist=True)
+    assert np.all(hist.sum(axis=1) == m)
+    h = 2.0 * value_range / bins
+    inside = np.abs(exact) < value_range - h
+    assert inside.sum() >= E // 2
+    assert np.max(np.abs(est[inside].astype(np.float64) - exact[inside])) < h * (1 + 1e-6)
+    # histogram = direct binning of the margins (numpy in binary32, same two rounded operations)
+    margin = oracle.sigmoid_f32(z) - alpha[:, None]
+    u = (margin + np.float32(value_range)) * (np.float32(bins) / (np.float32(2.0) * np.float32(value_range)))
+    k = np.clip(np.floor(u), 0, bins - 1).astype(np.int64)
+    for j in (0, E // 2, E - 1):
+        np.testing.assert_array_equal(hist[j], np.bincount(k[:, j], minlength=bins))
+
+
+def test_quantile_histogram_estimate_converges_to_the_exact_target():
+    rng = np.random.default_rng(62)
+    m, E, K = 300, 16, 2
+    z = (rng.standard_normal((m, E))).astype(np.float32)
+    _, _, alpha = oracle.route_f32(z, np.zeros(E, np.float32), K)
+    exact = oracle.quantile_target(z, alpha, K).astype(np.float64)
+    errs = [np.max(np.abs(oracle.quantile_target_hist(z, alpha, K, B, 1.0).astype(np.float64) - exact))
+            for B in (16, 256, 4096, 65536, 1 << 20)]
+    assert all(e < 2.0 / B * 1.000001 for e, B in zip(errs, (16, 256, 4096, 65536, 1 << 20)))
+    assert errs[-1] < 2e-6 and errs[-1] < errs[0]
+
+
 # ----------------------------------------------------------------- metrics
 @pytest.mark.parametrize("row", _rows("violation_bounds.txt"))
 def test_violation_bounds(row):
