@@ -237,10 +237,16 @@ def run_aux(args, wl):
     out["route_plus_quantile_update_us"] = {"median": med, "best": best}
     out["quantile_update_us"] = {"median": med - r_med, "note": "difference of the two lines above",
                                  "dump_GBps": 4 * dump_bytes / max(1e-9, (med - r_med)) / 1e3}
-    if hasattr(rs, "quantile_target_hist"):
-        tgt = torch.empty(wl.E, device=dev)
-        med, best = timed(lambda: rs.quantile_target_hist(logits[0], alpha[0], tgt), reps)
-        out["quantile_target_hist_us"] = {"median": med, "best": best, "dump_GBps": dump_bytes / best / 1e3}
+    rqh = binding.Router(1, wl.E, wl.K, wl.H, wl.T, controller="quantile", qb_hist_bins=1024, device=dev)
+
+    def qbh_route():
+        rqh.route_step(xs[state["i"] % 4], w, logits_out=logits, alpha_out=alpha)
+        state["i"] += 1
+    med_h, _ = timed(lambda: (qbh_route(), rqh.controller_update()), reps)
+    out["quantile_update_histogram_estimate_us"] = {
+        "median": med_h - r_med, "note": "1024-bin margin histogram, one pass over the dump; difference to the routing call",
+        "dump_GBps": dump_bytes / max(1e-9, (med_h - r_med)) / 1e3}
+    rqh.poll()
     rs.controller_update()
     idx, gate = rs.route_step(xs[0], w, logits_out=logits)
     loads = rs.loads_peek()

@@ -94,6 +94,15 @@ typedef struct {
                            the same time (the tile is streamed from HBM once) and a merge kernel finishes the
                            rows from L*ceil(E/256)*max_tokens*(K+1)*8 bytes of workspace; 0 = chosen by the
                            hidden size (2 when the tiles of all resident pairs no longer fit in L2) */
+  int32_t qb_hist_bins; /* MOE_CTRL_QUANTILE only.  0 = exact quantile of Eq. 7 (radix select over the dump).
+                           B > 0 (multiple of 32, 32..2048) = the estimate the footnote to Eq. 7 mentions for use
+                           at scale, from a per-expert margin histogram -- the paper fixes neither bins nor
+                           rule, this library uses B uniform bins over [-qb_hist_range, qb_hist_range) (margins
+                           outside count in the end bins), the same rank r = m - floor(mK/E), and linear
+                           interpolation inside the bin that holds the r-th smallest margin:
+                           estimate = -range + (k + ((r - below) - 0.5) / count_k) * (2 range / B).
+                           |estimate - exact| < 2 range / B while the exact value is inside the range. */
+  float qb_hist_range;  /* > 0; default 1 */
 } moe_route_config;
 
 /* Fills *cfg with the paper's defaults (Ki = Kd = 6e-3, eta = 1e-3, rho = 0,

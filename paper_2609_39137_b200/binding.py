@@ -32,7 +32,8 @@ class MoeRouteConfig(C.Structure):
                 ("top_k", C.c_int32), ("hidden", C.c_int32), ("max_tokens", C.c_int32), ("controller", C.c_int32),
                 ("ki", C.c_float), ("kd", C.c_float), ("eta", C.c_float), ("qb_ema_rho", C.c_float),
                 ("center", C.c_int32), ("spin_limit", C.c_int32), ("host_staging", C.c_int32),
-                ("w_layout", C.c_int32), ("chunk_split", C.c_int32)]
+                ("w_layout", C.c_int32), ("chunk_split", C.c_int32),
+                ("qb_hist_bins", C.c_int32), ("qb_hist_range", C.c_float)]
 
 
 class MoeRouteError(RuntimeError):
@@ -128,7 +129,7 @@ class Router:
 
     def __init__(self, num_layers, num_experts, top_k, hidden, max_tokens, controller="id", ki=None, kd=None,
                  eta=None, qb_ema_rho=None, center=None, spin_limit=0, host_staging=False, w_layout=0,
-                 chunk_split=0, device="cuda"):
+                 chunk_split=0, qb_hist_bins=0, qb_hist_range=None, device="cuda"):
         self.lib = load()
         cfg = default_config(num_layers, num_experts, top_k, hidden, max_tokens)
         cfg.controller = CONTROLLERS[controller] if isinstance(controller, str) else int(controller)
@@ -141,6 +142,8 @@ class Router:
         cfg.host_staging = int(bool(host_staging))
         cfg.w_layout = int(w_layout)
         cfg.chunk_split = int(chunk_split)
+        cfg.qb_hist_bins = int(qb_hist_bins)
+        if qb_hist_range is not None: cfg.qb_hist_range = float(qb_hist_range)
         self.cfg = cfg
         self.L, self.E, self.K, self.H, self.max_tokens = num_layers, num_experts, top_k, hidden, max_tokens
         self.device = torch.device(device)

@@ -63,12 +63,14 @@ Layout make_layout(const moe_route_config& c) {
   l.gate_count = take((size_t)c.num_layers * 4);
   l.qb_target = take(LE * 4);
   if (c.controller == MOE_CTRL_QUANTILE) {
-    l.qb_hist = take((size_t)c.num_experts * 256 * 4);
+    // exact selection: radix histogram [E][256]; histogram estimate: margin histogram [E][qb_hist_bins]
+    l.qb_hist = take((size_t)c.num_experts * (c.qb_hist_bins > 0 ? c.qb_hist_bins : 256) * 4);
     l.qb_prefix = take((size_t)c.num_experts * 4);
     l.qb_rank = take((size_t)c.num_experts * 4);
   }
   l.state_end = o;
-  if (c.controller == MOE_CTRL_QUANTILE) l.qb_keys = take((size_t)c.max_tokens * c.num_experts * 4);
+  if (c.controller == MOE_CTRL_QUANTILE && c.qb_hist_bins == 0)
+    l.qb_keys = take((size_t)c.max_tokens * c.num_experts * 4);
   {
     const size_t LC = (size_t)c.num_layers * stat_ctas_per_layer(c.num_layers);
     l.stat_P = take(LC * c.num_experts * 4);
@@ -106,6 +108,9 @@ bool config_ok(const moe_route_config* c) {
   if (c->spin_limit < 0) return false;
   if (c->w_layout != 0 && c->w_layout != 1) return false;
   if (c->chunk_split < 0 || c->chunk_split > 2) return false;
+  if (c->qb_hist_bins != 0 && (c->qb_hist_bins < 32 || c->qb_hist_bins > kQhMaxBins || (c->qb_hist_bins % 32) != 0))
+    return false;
+  if (c->qb_hist_bins != 0 && !(c->qb_hist_range > 0.0f && c->qb_hist_range <= 1e6f)) return false;
   return true;
 }
 
@@ -316,6 +321,8 @@ void moe_route_default_config(moe_route_config* cfg, int32_t num_layers, int32_t
   cfg->host_staging = 0;
   cfg->w_layout = 0;
   cfg->chunk_split = 0;
+  cfg->qb_hist_bins = 0;
+  cfg->qb_hist_range = 1.0f;
 }
 
 size_t moe_route_workspace_bytes(const moe_route_config* cfg) {
@@ -422,13 +429,46 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
   ctx->last_stream = st;
   if (c.controller == MOE_CTRL_QUANTILE) {
     if (!ctx->qb_logits) return fail(ctx, MOE_ERR_STATE, "quantile controller: no routing step since the last update");
+    if (c.qb_hist_bins > 0) {
+      // footnote to Eq. 7: the target estimated from a per-expert margin histogram, one pass over the dump
+      const size_t smem = (size_t)c.qb_hist_bins * kQhCols * 4;
+      static bool attr_set[64] = {};
+      if (!attr_set[ctx->device & 63]) {
+        cudaError_t ae = cudaFuncSetAttribute(qb_margin_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              kQhMaxBins * kQhCols * 4);
+        if (ae != cudaSuccess) return cuda_fail(ctx, ae, "cudaFuncSetAttribute(qb_margin_hist_kernel)");
+        attr_set[ctx->device & 63] = true;
+      }
+      const int groups = (c.num_experts + kQhCols - 1) / kQhCols;
+      const int per_sm = smem <= 32768 ? 6 : smem <= 65536 ? 3 : 1;
+      int splits = (per_sm * ctx->num_sms + groups - 1) / groups;
+      const int max_splits = (ctx->qb_tokens + 127) / 128;
+      if (splits > max_splits) splits = max_splits;
+      if (splits < 1) splits = 1;
+      for (int l = 0; l < c.num_layers; ++l) {
+        QhParams q{};
+        q.logits = ctx->qb_logits + (size_t)l * ctx->qb_tokens * c.num_experts;
+        q.alpha = ctx->qb_alpha + (size_t)l * ctx->qb_tokens;
+        q.m = ctx->qb_tokens; q.E = c.num_experts; q.K = c.top_k; q.B = c.qb_hist_bins;
+        q.range = c.qb_hist_range;
+        q.inv_h = (float)c.qb_hist_bins / (2.0f * c.qb_hist_range);
+        q.hist = at<uint32_t>(ctx, ctx->lay.qb_hist);
+        q.target = at<float>(ctx, ctx->lay.qb_target) + (size_t)l * c.num_experts;
+        qb_margin_hist_kernel<<<dim3(groups, splits), kQhThreads, smem, st>>>(q);
+        qb_margin_hist_finish_kernel<<<(c.num_experts * 32 + 255) / 256, 256, 0, st>>>(q);
+        ctx->launches += 2;
+      }
+      cudaError_t qe = cudaGetLastError();
+      if (qe != cudaSuccess) return cuda_fail(ctx, qe, "margin histogram kernels launch");
+      ctx->qb_logits = nullptr;
+    }
     const int col_groups = (c.num_experts + kQbCols - 1) / kQbCols;
     int splits = (6 * ctx->num_sms + col_groups - 1) / col_groups;
     const int max_splits = (ctx->qb_tokens + 63) / 64;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
     // Eq. 7 is per layer: the layers take turns on the one radix-select scratch (same stream, so in order)
-    for (int l = 0; l < c.num_layers; ++l) {
+    for (int l = 0; c.qb_hist_bins == 0 && l < c.num_layers; ++l) {
       QbParams q{};
       q.logits = ctx->qb_logits + (size_t)l * ctx->qb_tokens * c.num_experts;
       q.alpha = ctx->qb_alpha + (size_t)l * ctx->qb_tokens;

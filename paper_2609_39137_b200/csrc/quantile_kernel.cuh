@@ -168,4 +168,117 @@ __global__ void qb_scan_kernel(QbParams p, int pass) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// Quantile target estimated from a per-expert margin histogram (footnote to
+// Eq. 7: the estimate the paper mentions for use "at scale"; bins, range and
+// the rule inside a bin are this library's choice).  One pass over the dump:
+//   bin k = floor((d + range) * inv_h) clamped to [0, B-1], d = sigmoid(z) - alpha
+//   (two rounded binary32 operations), B uniform bins over [-range, range);
+// the counts of a CTA's 16 experts are kept in shared memory ([bin][expert]) and
+// flushed with one global atomic per non-empty bin.  A second kernel (one warp
+// per expert) finds the bin k* of the r-th smallest margin, r = m - floor(mK/E),
+// and interpolates in binary64: est = -range + (k* + ((r - below) - 0.5) / cnt) * h.
+// The counts are integers, so histograms of several ranks can be added before
+// the second kernel runs (that is what makes the estimate usable when the
+// tokens of a step are spread over data-parallel ranks).
+constexpr int kQhCols = 16;        // experts per CTA
+constexpr int kQhThreads = 256;
+constexpr int kQhRowsInFlight = 8;
+constexpr int kQhMaxBins = 2048;   // 16 experts x 2048 bins x 4 bytes = 128 KB of shared memory
+
+struct QhParams {
+  const float* logits;  // [m][E]
+  const float* alpha;   // [m]
+  int m, E, K, B;
+  float range, inv_h;   // inv_h = (float)B / (2 * range)
+  uint32_t* hist;       // [E][B], zero on entry of the histogram kernel, cleared again by the finish kernel
+  float* target;        // [E] out: Q_j
+};
+
+__device__ __forceinline__ int margin_bin(float d, float range, float inv_h, int B) {
+  const float u = __fmul_rn(__fadd_rn(d, range), inv_h);
+  if (!(u >= 0.0f)) return 0;
+  const float fl = floorf(u);
+  return (fl >= (float)B) ? B - 1 : (int)fl;
+}
+
+// grid = (ceil(E / 16), row_splits); dynamic shared memory B * 16 * 4 bytes.  A warp covers two rows of 16
+// experts (64 bytes each) per load; kQhRowsInFlight loads are issued before the first is used.
+__global__ void __launch_bounds__(kQhThreads) qb_margin_hist_kernel(QhParams p) {
+  extern __shared__ uint32_t hs[];   // [bin][col]
+  for (int i = threadIdx.x; i < p.B * kQhCols; i += kQhThreads) hs[i] = 0u;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = lane & (kQhCols - 1), sub = lane >> 4;
+  const int col = blockIdx.x * kQhCols + c;
+  const bool live = col < p.E;
+  const int rows_per = (p.m + gridDim.y - 1) / gridDim.y;
+  const int r0 = blockIdx.y * rows_per;
+  const int r1 = min(p.m, r0 + rows_per);
+  constexpr int kRowsPerIter = (kQhThreads / 32) * 2;   // rows taken by the CTA per load
+  for (int i0 = r0 + warp * 2 + sub; i0 < r1; i0 += kRowsPerIter * kQhRowsInFlight) {
+    float z[kQhRowsInFlight], a[kQhRowsInFlight];
+#pragma unroll
+    for (int u = 0; u < kQhRowsInFlight; ++u) {
+      const int i = i0 + u * kRowsPerIter;
+      const bool ok = live && i < r1;
+      z[u] = ok ? __ldg(p.logits + (size_t)i * p.E + col) : 0.0f;
+      a[u] = ok ? __ldg(p.alpha + i) : 0.0f;
+    }
+#pragma unroll
+    for (int u = 0; u < kQhRowsInFlight; ++u) {
+      const int i = i0 + u * kRowsPerIter;
+      if (live && i < r1) {
+        const float d = __fsub_rn(sigmoid_score(z[u]), a[u]);
+        atomicAdd(&hs[margin_bin(d, p.range, p.inv_h, p.B) * kQhCols + c], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < p.B * kQhCols; i += kQhThreads) {
+    const int cc = blockIdx.x * kQhCols + (i & (kQhCols - 1));
+    const uint32_t cnt = hs[i];
+    if (cnt != 0u && cc < p.E) atomicAdd(&p.hist[(size_t)cc * p.B + (i >> 4)], cnt);
+  }
+}
+
+// One warp per expert: lane l owns the bins [l * B/32, (l+1) * B/32) (B is a multiple of 32).
+__global__ void qb_margin_hist_finish_kernel(QhParams p) {
+  const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (j >= p.E) return;
+  uint32_t* hj = p.hist + (size_t)j * p.B;
+  const int per = p.B / 32;
+  uint32_t mine = 0;
+  for (int t = 0; t < per; ++t) mine += hj[lane * per + t];
+  uint32_t incl = mine;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += o;
+  }
+  long long r = (long long)p.m - ((long long)p.m * p.K) / p.E;
+  if (r < 1) r = 1;
+  if (r > p.m) r = p.m;
+  const uint32_t rank = (uint32_t)r;
+  const uint32_t excl = incl - mine;
+  if (rank > excl && rank <= incl) {           // exactly one lane: the counts of an expert sum to m >= rank
+    uint32_t run = excl;
+    for (int t = 0; t < per; ++t) {
+      const uint32_t cnt = hj[lane * per + t];
+      if (rank <= run + cnt) {
+        const int kstar = lane * per + t;
+        const double h = __ddiv_rn(__dmul_rn(2.0, (double)p.range), (double)p.B);
+        const double inside = __ddiv_rn(__dsub_rn((double)(rank - run), 0.5), (double)cnt);
+        const double est = __dadd_rn(-(double)p.range, __dmul_rn(__dadd_rn((double)kstar, inside), h));
+        p.target[j] = -(float)est;
+        break;
+      }
+      run += cnt;
+    }
+  }
+  __syncwarp();
+  for (int t = 0; t < per; ++t) hj[lane * per + t] = 0u;   // ready for the next update
+}
+
 }  // namespace moe

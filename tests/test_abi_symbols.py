@@ -27,7 +27,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_config_struct_matches_header(lib):
     cfg = binding.default_config(2, 768, 10, 2048, 16384)
-    assert cfg.struct_size == C.sizeof(binding.MoeRouteConfig) == 16 * 4
+    assert cfg.struct_size == C.sizeof(binding.MoeRouteConfig) == 18 * 4
     # paper defaults: Ki = Kd = 6e-3 (Section 4), eta = 1e-3 (Section 4.1), no EMA
     assert abs(cfg.ki - 6e-3) < 1e-9 and abs(cfg.kd - 6e-3) < 1e-9 and abs(cfg.eta - 1e-3) < 1e-9
     assert cfg.qb_ema_rho == 0 and cfg.center == -1 and cfg.controller == binding.MOE_CTRL_ID
@@ -41,7 +41,8 @@ def test_workspace_bytes_and_config_validation(lib):
     assert lib.moe_route_workspace_bytes(C.byref(cfg)) > n + 48 * 16384 * 2048 * 2
     bad = [dict(num_experts=770), dict(num_experts=2048), dict(top_k=0), dict(top_k=17), dict(hidden=100),
            dict(num_layers=0), dict(max_tokens=0), dict(controller=7), dict(qb_ema_rho=1.0), dict(ki=-1.0),
-           dict(struct_size=8), dict(w_layout=2), dict(chunk_split=3)]
+           dict(struct_size=8), dict(w_layout=2), dict(chunk_split=3), dict(qb_hist_bins=48),
+           dict(qb_hist_bins=4096), dict(qb_hist_bins=64, qb_hist_range=0.0)]
     for kw in bad:
         c = binding.default_config(48, 768, 10, 2048, 16384)
         for k, v in kw.items():

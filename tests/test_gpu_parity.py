@@ -318,6 +318,34 @@ def test_quantile_controller_at_full_single_layer_size(K):
     assert 0 <= hist[0][0] <= wl.E / K - 1 + 1e-4
 
 
+@pytest.mark.parametrize("bins,value_range,T,L", [(1024, 1.0, 3000, 1), (64, 0.5, 700, 2), (2048, 2.0, 16384, 1)])
+def test_quantile_controller_with_margin_histogram_estimate(bins, value_range, T, L):
+    # footnote to Eq. 7: the target estimated from a per-expert margin histogram (this library's bin rule).
+    # Integer counts and a fixed binary64 interpolation: bit-exact against the oracle's estimate on the GPU's own
+    # dump, and within one bin width of the exact target wherever that lies inside the range
+    wl = synth.WORKLOADS["top3_single"].with_(T=T, H=256, L=L)
+    dev = "cuda"
+    r = binding.Router(L, wl.E, wl.K, wl.H, wl.T, controller="quantile", qb_hist_bins=bins, qb_hist_range=value_range)
+    w = torch.stack([synth.router_weights(wl, l, dev) for l in range(L)])
+    logits = torch.empty(L, wl.T, wl.E, device=dev)
+    alpha = torch.empty(L, wl.T, device=dev)
+    for step in range(2):                      # the second update starts from a histogram the first one cleared
+        x = torch.stack([synth.hidden_states(wl, l, step, dev) for l in range(L)])
+        r.route_step(x, w, logits_out=logits, alpha_out=alpha)
+        r.controller_update()
+        r.poll()
+        bias = np_(r.load_stats()[1])
+        for l in range(L):
+            lg, al = np_(logits)[l], np_(alpha)[l]
+            want = oracle.quantile_target_hist(lg, al, wl.K, bins, value_range)
+            np.testing.assert_array_equal(bits(bias[l]), bits(want))
+            exact = oracle.quantile_target(lg, al, wl.K)
+            h = 2.0 * value_range / bins
+            inside = np.abs(exact) < value_range - h
+            assert inside.sum() > wl.E // 2
+            assert np.max(np.abs(bias[l][inside].astype(np.float64) - exact[inside])) < h * (1 + 1e-6)
+
+
 def test_closed_loop_drifting_deep_stack_opens_the_derivative_gate():
     # deep-stack configuration at a reduced token count: the cluster means drift linearly over the 500 steps of
     # the workload, so consecutive controller steps taken from steps spread over the drift see the imbalance of
