@@ -58,7 +58,9 @@ enum {
   MOE_ERR_CUDA = 3,
   MOE_ERR_STATE = 4,      /* e.g. controller update with no tokens routed */
   MOE_ERR_WORKSPACE = 5,  /* workspace too small or misaligned */
-  MOE_ERR_TIMEOUT = 6     /* a bounded device-side wait expired */
+  MOE_ERR_TIMEOUT = 6,    /* a bounded device-side wait expired */
+  MOE_ERR_INTERNAL = 7    /* builds with -DMOE_DEBUG only: an index guard inside a kernel tripped (the access
+                             was skipped) or a canary between two workspace sections was overwritten */
 };
 
 enum {
@@ -286,6 +288,13 @@ int moe_debug_wait_timeout(moe_route_ctx* ctx, int32_t spin_limit, void* cuda_st
  * of every CTA leaves its loop, tensor memory is released, the kernel returns,
  * and moe_route_poll reports MOE_ERR_TIMEOUT.  Host call; nothing is enqueued. */
 int moe_debug_route_stall(moe_route_ctx* ctx, int32_t after_loads);
+
+/* 1 if the library was compiled with -DMOE_DEBUG, else 0.  That build is the stand-in for a memory checker:
+ * the routing kernel guards the indices of its shared-memory log, exchange area, output and candidate
+ * writes (a bad index is recorded and the access skipped), every workspace section is followed by a
+ * 256-byte canary, and moe_route_poll reports either as MOE_ERR_INTERNAL.  Results are identical to the
+ * release build's; moe_route_workspace_bytes is larger by the canaries. */
+int moe_debug_build(void);
 
 /* Number of kernels this context has launched so far. */
 int64_t moe_route_launch_count(const moe_route_ctx* ctx);

@@ -12,9 +12,11 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmoe_route_b200.so")
+# MOE_ROUTE_LIB selects another build of the same library (the -DMOE_DEBUG one, libmoe_route_b200_debug.so)
+LIB_PATH = os.environ.get("MOE_ROUTE_LIB") or os.path.join(_HERE, "libmoe_route_b200.so")
 
-MOE_OK, MOE_ERR_INVALID_ARG, MOE_ERR_UNSUPPORTED, MOE_ERR_CUDA, MOE_ERR_STATE, MOE_ERR_WORKSPACE, MOE_ERR_TIMEOUT = range(7)
+(MOE_OK, MOE_ERR_INVALID_ARG, MOE_ERR_UNSUPPORTED, MOE_ERR_CUDA, MOE_ERR_STATE, MOE_ERR_WORKSPACE, MOE_ERR_TIMEOUT,
+ MOE_ERR_INTERNAL) = range(8)
 MOE_CTRL_ID, MOE_CTRL_FIXED_STEP, MOE_CTRL_QUANTILE, MOE_CTRL_FROZEN = range(4)
 CONTROLLERS = {"id": MOE_CTRL_ID, "fixed_step": MOE_CTRL_FIXED_STEP, "quantile": MOE_CTRL_QUANTILE,
                "frozen": MOE_CTRL_FROZEN}
@@ -24,7 +26,7 @@ SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_i
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_loads_buffer", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
            "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_quantile_target_static",
-           "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout", "moe_score_stats", "moe_debug_route_stall"]
+           "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout", "moe_score_stats", "moe_debug_route_stall", "moe_debug_build"]
 
 
 class MoeRouteConfig(C.Structure):
@@ -81,6 +83,7 @@ def load():
     L.moe_debug_score_gap.argtypes = [vp, vp]
     L.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
     L.moe_debug_route_stall.argtypes = [vp, i32]
+    L.moe_debug_build.argtypes = []
     L.moe_score_stats.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.moe_quantile_target_static.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     _lib = L

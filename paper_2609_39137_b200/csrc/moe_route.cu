@@ -34,7 +34,15 @@ struct Layout {
   size_t w_t;   // [L][E][H] bf16 copy of the weights when they are given as [L][H][E]
   size_t cand;  // [L][chunks][max_tokens][K+1] (score, expert) pairs, chunk-split scheduling only
   size_t total;
+#ifdef MOE_DEBUG
+  // debug build: every section is followed by a 256-byte canary that moe_route_poll checks
+  int num_guards;
+  size_t guard[48];
+#endif
 };
+#ifdef MOE_DEBUG
+constexpr unsigned char kCanaryByte = 0xC5;
+#endif
 
 // Chunk-split scheduling (the expert chunks of a token tile go to different CTA pairs, a merge kernel
 // finishes): chosen when one CTA pair re-reading its tile once per chunk would push the tiles of all
@@ -51,7 +59,17 @@ Layout make_layout(const moe_route_config& c) {
   Layout l{};
   size_t o = 0;
   const size_t LE = (size_t)c.num_layers * c.num_experts;
+#ifdef MOE_DEBUG
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    o = align_up(o + bytes);
+    if (l.num_guards < 48) l.guard[l.num_guards++] = o;
+    o += kAlign;
+    return at;
+  };
+#else
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+#endif
   l.status = take(64);
   l.bias = take(LE * 4);
   l.e_prev = take(LE * 4);
@@ -356,6 +374,10 @@ int moe_route_init(const moe_route_config* cfg, void* dev_workspace, size_t work
   if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) { delete ctx; return MOE_ERR_CUDA; }
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   e = cudaMemset(dev_workspace, 0, lay.state_end);
+#ifdef MOE_DEBUG
+  for (int g = 0; g < lay.num_guards && e == cudaSuccess; ++g)
+    e = cudaMemset(static_cast<uint8_t*>(dev_workspace) + lay.guard[g], kCanaryByte, kAlign);
+#endif
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) { delete ctx; return MOE_ERR_CUDA; }
   *out = ctx;
@@ -685,6 +707,17 @@ int moe_route_poll(moe_route_ctx* ctx) {
   int st[2] = {0, 0};
   e = cudaMemcpy(st, status_ptr(ctx), sizeof st, cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "status read");
+#ifdef MOE_DEBUG
+  for (int g = 0; g < ctx->lay.num_guards && st[0] == MOE_OK; ++g) {
+    unsigned char canary[kAlign];
+    if (cudaMemcpy(canary, ctx->ws + ctx->lay.guard[g], kAlign, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return cuda_fail(ctx, cudaGetLastError(), "canary read");
+    for (size_t i = 0; i < kAlign; ++i)
+      if (canary[i] != kCanaryByte)
+        return fail(ctx, MOE_ERR_INTERNAL, "workspace canary %d (offset %zu) overwritten at byte %zu", g,
+                    ctx->lay.guard[g], i);
+  }
+#endif
   if (st[0] != MOE_OK) {
     cudaMemset(status_ptr(ctx), 0, sizeof st);
     if (st[0] == MOE_ERR_TIMEOUT) {
@@ -696,6 +729,8 @@ int moe_route_poll(moe_route_ctx* ctx) {
     }
     if (st[0] == MOE_ERR_STATE)
       return fail(ctx, MOE_ERR_STATE, "controller update on a layer with no routed tokens");
+    if (st[0] == MOE_ERR_INTERNAL)
+      return fail(ctx, MOE_ERR_INTERNAL, "debug build: index guard %d of the routing kernel tripped", st[1] - 1000);
     return fail(ctx, st[0], "device status %d", st[0]);
   }
   return MOE_OK;
@@ -826,6 +861,14 @@ int moe_quantile_target_static(const float* logits, const float* alpha, int32_t 
     qb_scan_kernel<<<(num_experts * 32 + 255) / 256, 256, 0, st>>>(q, pass);
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+int moe_debug_build(void) {
+#ifdef MOE_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
 }
 
 int64_t moe_route_launch_count(const moe_route_ctx* ctx) { return ctx ? ctx->launches : 0; }
