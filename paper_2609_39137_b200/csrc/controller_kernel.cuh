@@ -195,35 +195,70 @@ struct DiagParams {
 };
 
 __global__ void __launch_bounds__(kCtrlThreads) diagnostics_kernel(const DiagParams p) {
-  __shared__ int n_s[kCtrlThreads];
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned int sel_prefix, sel_rank;
   __shared__ long long red_a[32], red_b[32];
-  __shared__ int red_c[32];
+  __shared__ int red_c[32], red_d[32];
   __shared__ double y[kCtrlThreads];
   const int layer = blockIdx.x, i = threadIdx.x, lane = i & 31, warp = i >> 5;
   const bool live = i < p.E;
   const size_t o = (size_t)layer * p.E + i;
   const int n = live ? p.loads_last[o] : -1;
-  n_s[i] = n;
   y[i] = live ? fabs((double)p.bias[o] - (double)p.bias_prev[o]) : 0.0;
-  __syncthreads();
-  // rank of expert i by load (descending, ties by index): the m best ranks are the busiest experts
-  int rank = 0;
-  if (live)
-    for (int j = 0; j < p.E; ++j) {
-      const int nj = n_s[j];
-      rank += (nj > n) || (nj == n && j < i);
-    }
+  // The share of the busiest m experts needs the sum of the m largest loads: the m-th largest load v* is
+  // found by a radix select (four 8-bit digits, most significant first, shared-memory histogram of the
+  // values that still match the digits fixed so far); the sum is then that of the loads above v* plus
+  // v* for the remaining places -- equal loads are interchangeable, so no order among them is needed.
   int m = (p.E + 5) / 10;
   if (m < 1) m = 1;
-  long long tot = live ? n : 0, top = (live && rank < m) ? n : 0;
+  const unsigned int key = live ? (unsigned int)n : 0u;        // loads are non-negative
+  if (i == 0) { sel_prefix = 0u; sel_rank = (unsigned int)m; }
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (i < 256) hist[i] = 0u;
+    __syncthreads();
+    const unsigned int pre = sel_prefix;
+    if (live && (pass == 0 || ((key ^ pre) >> (shift + 8)) == 0u)) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    __syncthreads();
+    if (warp == 0) {
+      // lane l owns bins 255 - 8l ... 248 - 8l (descending): find the bin where the count from the top reaches the rank
+      unsigned int c[8], mine = 0;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { c[t] = hist[255 - (lane * 8 + t)]; mine += c[t]; }
+      unsigned int incl = mine;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const unsigned int up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+      }
+      const unsigned int rank = sel_rank, excl = incl - mine;
+      if (rank > excl && rank <= incl) {
+        unsigned int run = excl;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          if (rank > run && rank <= run + c[t]) {
+            sel_prefix = pre | ((unsigned int)(255 - (lane * 8 + t)) << shift);
+            sel_rank = rank - run;
+          }
+          run += c[t];
+        }
+      }
+    }
+    __syncthreads();
+  }
+  const int vstar = (int)sel_prefix;            // the m-th largest load
+  long long tot = live ? n : 0, top = (live && n > vstar) ? n : 0;
+  int above = (live && n > vstar) ? 1 : 0;
   int empty = (live && n == 0) ? 1 : 0;
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) {
     tot += __shfl_xor_sync(0xffffffffu, tot, d);
     top += __shfl_xor_sync(0xffffffffu, top, d);
     empty += __shfl_xor_sync(0xffffffffu, empty, d);
+    above += __shfl_xor_sync(0xffffffffu, above, d);
   }
-  if (lane == 0) { red_a[warp] = tot; red_b[warp] = top; red_c[warp] = empty; }
+  if (lane == 0) { red_a[warp] = tot; red_b[warp] = top; red_c[warp] = empty; red_d[warp] = above; }
   for (int stride = kCtrlThreads / 2; stride >= 1; stride >>= 1) {
     __syncthreads();
     if (i < stride) y[i] = __dadd_rn(y[i], y[i + stride]);
@@ -231,8 +266,9 @@ __global__ void __launch_bounds__(kCtrlThreads) diagnostics_kernel(const DiagPar
   __syncthreads();
   if (i == 0) {
     long long t = 0, tp = 0;
-    int em = 0;
-    for (int w = 0; w < kCtrlThreads / 32; ++w) { t += red_a[w]; tp += red_b[w]; em += red_c[w]; }
+    int em = 0, ab = 0;
+    for (int w = 0; w < kCtrlThreads / 32; ++w) { t += red_a[w]; tp += red_b[w]; em += red_c[w]; ab += red_d[w]; }
+    tp += (long long)(m - ab) * vstar;          // the places among the m busiest that are held by loads equal to v*
     float* out = p.out + (size_t)layer * 4;
     out[0] = (float)__ddiv_rn((double)p.gate_count[layer], (double)p.E);
     out[1] = t > 0 ? (float)__ddiv_rn((double)tp, (double)t) : 0.0f;
