@@ -160,6 +160,8 @@ struct moe_route_ctx {
   int64_t launches;
   int64_t ctrl_steps;   // controller updates enqueued so far (exported / restored with the controller state)
   int stall_next;       // moe_debug_route_stall: applies to the next routing launch only
+  size_t merge_occ_smem;   // resident CTAs per SM of route_merge_kernel, cached per shared-memory size
+  int merge_occ;
   // cached TMA descriptors
   const void* map_x_ptr;
   const void* map_w_ptr;
@@ -299,10 +301,34 @@ int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, in
   mp.T = T; mp.E = c.num_experts; mp.K = c.top_k; mp.num_chunks = rp.num_chunks; mp.cand_len = need;
   mp.cand = rp.cand; mp.bias = rp.bias; mp.loads = rp.loads;
   mp.topk_idx = idx; mp.topk_gate = gate; mp.alpha_out = alpha;
+  {
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+      cudaError_t ae = cudaFuncSetAttribute(route_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)merge_smem_bytes(kMergeMaxChunks * (kMergeMaxK + 1)));
+      if (ae != cudaSuccess) return cuda_fail(ctx, ae, "cudaFuncSetAttribute(route_merge_kernel)");
+      attr_set[ctx->device & 63] = true;
+    }
+  }
+  // a CTA walks tokens of one layer and flushes its histogram once; the grid is at most what is resident at
+  // once (a grid slightly above that would run a second, almost empty wave)
+  const size_t merge_smem = merge_smem_bytes(rp.num_chunks * need);
+  if (ctx->merge_occ < 1 || ctx->merge_occ_smem != merge_smem) {
+    int occ = 0;
+    cudaError_t oe = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, route_merge_kernel, kMergeThreads, merge_smem);
+    if (oe != cudaSuccess || occ < 1) return cuda_fail(ctx, oe, "occupancy of route_merge_kernel");
+    ctx->merge_occ = occ;
+    ctx->merge_occ_smem = merge_smem;
+  }
+  const int per_sm = ctx->merge_occ;
+  const int num_tiles = (T + kMergeThreads - 1) / kMergeThreads;
+  int slices = (per_sm * ctx->num_sms) / c.num_layers;
+  if (slices > num_tiles) slices = num_tiles;
+  if (slices < 1) slices = 1;
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3((T + kMergeRowsPerCta - 1) / kMergeRowsPerCta, c.num_layers);
+  lc.gridDim = dim3(slices, c.num_layers);
   lc.blockDim = dim3(kMergeThreads);
-  lc.dynamicSmemBytes = 0;
+  lc.dynamicSmemBytes = merge_smem;
   lc.stream = st;
   cudaLaunchAttribute attr{};
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;

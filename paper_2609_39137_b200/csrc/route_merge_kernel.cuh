@@ -1,18 +1,28 @@
 // Second half of a routing step under chunk-split scheduling.
 //
-// When the token tiles are long (hidden > 2048) the routing kernel gives the
-// expert chunks of one tile to different CTA pairs that run at the same time,
-// so the tile is streamed from HBM once and the other readers find it in L2.
-// Each (tile, chunk) item leaves, per token, its chunk's best `cand_len`
-// experts as (score s, expert e) pairs in ranking order (biased score
-// descending, expert ascending).  The chunks cover disjoint experts, so the
-// K best of the row (Eq. 2) are the first K of the merge of those sorted
-// lists: this kernel recomputes the biased score v = s + b_e (one rounded
-// addition, the same operation the routing kernel ordered by), merges, and
-// produces what the fused epilogue produces otherwise -- indices, gates
-// (selected scores normalised without the bias, sequential fp32 sum in output
-// order), alpha = rank K+1 on request, and the load histogram (Algorithm 1
-// line 4: shared-memory counts, one global atomic per non-zero expert per CTA).
+// When the token tiles are long the routing kernel gives the expert chunks of
+// one tile to different CTA pairs that run at the same time, so the tile is
+// streamed from HBM once and the other readers find it in L2.  Each (tile,
+// chunk) item leaves, per token, its chunk's best `cand_len` experts as
+// (score s, expert e) pairs in ranking order (biased score descending, expert
+// ascending); the lists of a token are contiguous: cand[layer][token][chunk][cand_len].
+// The chunks cover disjoint experts, so the K best of the row (Eq. 2) are the
+// first K of the merge of those sorted lists: this kernel recomputes the biased
+// score v = s + b_e (one rounded addition, the same operation the routing
+// kernel ordered by), merges, and produces what the fused epilogue produces
+// otherwise -- indices, gates (selected scores normalised without the bias,
+// sequential fp32 sum in output order), alpha = rank K+1 on request, and the
+// load histogram (Algorithm 1 line 4).
+//
+// Memory-bound: per token it reads num_chunks * cand_len * 8 bytes and writes
+// 8 K (+4) bytes.  A warp takes 32 consecutive tokens: their lists are one
+// contiguous block, which the lanes fetch with coalesced loads (batches of
+// independent loads in flight) into the warp's part of shared memory, one row
+// per token with an odd row stride (conflict-free both for the staging and for
+// the lanes reading different entries of their own rows); then each lane
+// merges its own token from there and stores its outputs.  A CTA walks tokens
+// of ONE layer and flushes its histogram once at its end (one global atomic per
+// non-zero expert per CTA); inside the token loop only warps synchronise.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -22,12 +32,13 @@
 namespace moe {
 
 constexpr int kMergeThreads = 256;
-constexpr int kMergeRowsPerCta = 1024;
 constexpr int kMergeMaxChunks = 4;     // 1024 experts / 256 per chunk
+constexpr int kMergeMaxK = 16;
+constexpr int kMergeBatch = 8;         // independent loads in flight per thread
 
 struct MergeParams {
   int T, E, K, num_chunks, cand_len;
-  const float2* cand;   // [L][num_chunks][T][cand_len]
+  const float2* cand;   // [L][T][num_chunks][cand_len]
   const float* bias;    // [L][E]
   int* loads;           // [L][E] accumulators (added to)
   int32_t* topk_idx;    // [L][T][K]
@@ -35,35 +46,67 @@ struct MergeParams {
   float* alpha_out;     // [L][T] or nullptr
 };
 
-// grid = (ceil(T / kMergeRowsPerCta), L); one thread per token row, kMergeRowsPerCta / kMergeThreads rows each
+// row stride of the staged lists in float2 units (odd)
+__host__ __device__ inline int merge_row_stride(int n_all) { return n_all | 1; }
+__host__ __device__ inline size_t merge_smem_bytes(int n_all) {
+  return (size_t)kMergeThreads * merge_row_stride(n_all) * sizeof(float2);
+}
+
+// grid = (slices, L); dynamic shared memory merge_smem_bytes(num_chunks * cand_len)
 __global__ void __launch_bounds__(kMergeThreads) route_merge_kernel(const MergeParams p) {
+  extern __shared__ float2 lists_s[];                       // [entry][thread]
   __shared__ float bias_s[1024];
   __shared__ int hist_s[1024];
   const int layer = blockIdx.y;
+  const int tid = threadIdx.x;
+  const int n_all = p.num_chunks * p.cand_len;
   // launched with programmatic stream serialisation behind the routing kernel: its lists are complete and
   // visible only after this wait
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  for (int i = threadIdx.x; i < 1024; i += kMergeThreads) {
+  for (int i = tid; i < 1024; i += kMergeThreads) {
     bias_s[i] = (i < p.E) ? p.bias[(size_t)layer * p.E + i] : -INFINITY;
     hist_s[i] = 0;
   }
   __syncthreads();
-  const int row_end = min(p.T, (int)(blockIdx.x + 1) * kMergeRowsPerCta);
-  for (int tok = blockIdx.x * kMergeRowsPerCta + threadIdx.x; tok < row_end; tok += kMergeThreads) {
-    // heads of the chunk lists
-    const float2* lst[kMergeMaxChunks];
+  const int lane = tid & 31;
+  const int stride = merge_row_stride(n_all);
+  float2* warp_s = lists_s + (size_t)(tid - lane) * stride;  // rows of this warp's 32 tokens
+  const float2* mine = warp_s + lane * stride;
+  const float uniform = __fdiv_rn(1.0f, (float)p.K);
+  // warp-uniform loop: tok0 = first token of the warp's group of 32
+  for (int tok0 = blockIdx.x * kMergeThreads + (tid - lane); tok0 < p.T; tok0 += gridDim.x * kMergeThreads) {
+    const int rows = min(32, p.T - tok0);
+    const int total = rows * n_all;                        // float2 elements of the group, contiguous
+    const float2* src = p.cand + ((size_t)layer * p.T + tok0) * n_all;
+    __syncwarp();                                          // the previous group's merges have read the rows
+    int r = 0, n = lane;                                   // element lane + 32 j as (row, entry)
+    while (n >= n_all) { n -= n_all; r += 1; }
+    const int dr = 32 / n_all, dn = 32 - dr * n_all;       // advancing the element by 32
+#pragma unroll 1
+    for (int i0 = lane; i0 < total + lane; i0 += 32 * kMergeBatch) {
+      float2 t[kMergeBatch];
+#pragma unroll
+      for (int u = 0; u < kMergeBatch; ++u)
+        t[u] = (i0 + 32 * u < total) ? __ldg(src + i0 + 32 * u) : make_float2(0.0f, 0.0f);
+#pragma unroll
+      for (int u = 0; u < kMergeBatch; ++u) {
+        if (i0 + 32 * u < total) warp_s[r * stride + n] = t[u];
+        r += dr; n += dn;
+        if (n >= n_all) { n -= n_all; r += 1; }
+      }
+    }
+    __syncwarp();
+    const int tok = tok0 + lane;
+    if (lane < rows) {
     float hv[kMergeMaxChunks], hs[kMergeMaxChunks];
     int he[kMergeMaxChunks], pos[kMergeMaxChunks];
 #pragma unroll
-    for (int c = 0; c < kMergeMaxChunks; ++c) {
-      pos[c] = (c < p.num_chunks) ? 0 : p.cand_len;       // a chunk that does not exist is an exhausted list
-      lst[c] = p.cand + (((size_t)layer * p.num_chunks + (c < p.num_chunks ? c : 0)) * p.T + tok) * p.cand_len;
-    }
+    for (int c = 0; c < kMergeMaxChunks; ++c) pos[c] = 0;
     auto load_head = [&](int c) {
       // an exhausted list, an entry without an expert and a padding column all rank after every real entry
       float2 se = make_float2(0.0f, __int_as_float(0x7fffffff));
-      if (pos[c] < p.cand_len) se = lst[c][pos[c]];
+      if (c < p.num_chunks && pos[c] < p.cand_len) se = mine[c * p.cand_len + pos[c]];
       const int e = __float_as_int(se.y);
       const bool real = (unsigned)e < (unsigned)p.E;
       hs[c] = se.x;
@@ -72,46 +115,59 @@ __global__ void __launch_bounds__(kMergeThreads) route_merge_kernel(const MergeP
     };
 #pragma unroll
     for (int c = 0; c < kMergeMaxChunks; ++c) load_head(c);
-    float sel_s[16];
-    int sel_e[16];
     float alpha = __int_as_float(0x7fc00000);
+    float denom = 0.0f;
+    float sel_s[kMergeMaxK];
+    int sel_e[kMergeMaxK];
 #pragma unroll
-    for (int k = 0; k < 17; ++k) {
-      if (k <= p.K) {           // rank K is only needed for alpha
+    for (int k = 0; k < kMergeMaxK + 1; ++k) {
+      if (k < p.cand_len) {                                // rank K is only needed for alpha
         int best = 0;
-#pragma unroll
-        for (int c = 1; c < kMergeMaxChunks; ++c)
-          if (ranks_before(hv[c], he[c], hv[best], he[best])) best = c;
         float bv = hv[0], bs = hs[0];
         int be = he[0];
 #pragma unroll
         for (int c = 1; c < kMergeMaxChunks; ++c)
-          if (best == c) { bv = hv[c]; bs = hs[c]; be = he[c]; }
-        if (k < 16 && k < p.K) { sel_s[k] = bs; sel_e[k] = be; }
+          if (ranks_before(hv[c], he[c], bv, be)) { best = c; bv = hv[c]; bs = hs[c]; be = he[c]; }
+        if (k < kMergeMaxK && k < p.K) {
+          sel_s[k] = bs;
+          sel_e[k] = be;
+          denom = (k == 0) ? bs : __fadd_rn(denom, bs);     // D = ((s_0 + s_1) + s_2) + ... in output order
+        }
         if (k == p.K) alpha = bv;
 #pragma unroll
         for (int c = 0; c < kMergeMaxChunks; ++c)
           if (best == c) { pos[c] += 1; load_head(c); }
       }
     }
-    float denom = sel_s[0];
+    // every entry of the row has been read: the row now takes the outputs, (expert, gate) at position k
+    float2* out_row = warp_s + lane * stride;
 #pragma unroll
-    for (int k = 1; k < 16; ++k)
-      if (k < p.K) denom = __fadd_rn(denom, sel_s[k]);
-    const float uniform = __fdiv_rn(1.0f, (float)p.K);
-    const size_t o = ((size_t)layer * p.T + tok) * p.K;
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
+    for (int k = 0; k < kMergeMaxK; ++k) {
       if (k < p.K) {
-        p.topk_idx[o + k] = sel_e[k];
-        p.topk_gate[o + k] = (denom == 0.0f) ? uniform : __fdiv_rn(sel_s[k], denom);
+        out_row[k] = make_float2(__int_as_float(sel_e[k]), (denom == 0.0f) ? uniform : __fdiv_rn(sel_s[k], denom));
         if ((unsigned)sel_e[k] < (unsigned)p.E) atomicAdd(&hist_s[sel_e[k]], 1);
       }
     }
     if (p.alpha_out != nullptr) p.alpha_out[(size_t)layer * p.T + tok] = alpha;
+    }   // lane < rows
+    __syncwarp();
+    // the group's outputs are contiguous in global memory (rows x K words): consecutive lanes, consecutive words
+    {
+      const size_t o0 = ((size_t)layer * p.T + tok0) * p.K;
+      int rr = 0, kk = lane;
+      while (kk >= p.K) { kk -= p.K; rr += 1; }
+      const int drr = 32 / p.K, dkk = 32 - drr * p.K;
+      for (int j = lane; j < rows * p.K; j += 32) {
+        const float2 eg = warp_s[rr * stride + kk];
+        p.topk_idx[o0 + j] = __float_as_int(eg.x);
+        p.topk_gate[o0 + j] = eg.y;
+        rr += drr; kk += dkk;
+        if (kk >= p.K) { kk -= p.K; rr += 1; }
+      }
+    }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < p.E; i += kMergeThreads) {
+  for (int i = tid; i < p.E; i += kMergeThreads) {
     const int n = hist_s[i];
     if (n != 0) atomicAdd(&p.loads[(size_t)layer * p.E + i], n);
   }
