@@ -51,7 +51,12 @@ L2_BYTES = 126e6
 # launch; the traffic of a launch with more layers of the same shape is scaled by the layer count (every layer
 # streams its own x once and re-reads nothing of another layer's).
 NCU_TRAFFIC = {
-    "top10_single": {"bytes": 70629376 + 1660928, "layers": 1, "profile": "profiles/route_step_kernel_top10_single.md"},
+    # routing kernel read + write, merge kernel read + write (2 of the 60 layers: a capture of the full launch
+    # would hold 64 GB on the device under the profiler)
+    "top10_large": {"bytes": 1142379000 + 79602176 + 31528448 + 512, "layers": 2,
+                    "profile": "profiles/route_step_kernel_top10_large.md"},
+    "top10_single": {"bytes": 71004416 + 2727680, "layers": 1, "profile": "profiles/route_step_kernel_top10_single.md"},
+    "top10_deep": {"bytes": 329675008 + 17733632, "layers": 4, "profile": "profiles/route_step_kernel_top10_deep_4layers.md"},
 }
 
 
@@ -389,7 +394,7 @@ def roofline_of(wl, total_ms, steps_total, route_ms, pk):
     else:
         traffic, traffic_note = None, "no ncu capture of this workload"
     algo_bytes = wl.L * (wl.T * wl.H * 2 + wl.E * wl.H * 2 + wl.T * wl.K * 8)
-    return {"kernel": "route_step_kernel", "bound": "tensor", "achieved": achieved, "peak": pk["tflops"],
+    return {"kernel": "route_step_kernel (+ route_merge_kernel under chunk-split scheduling)", "bound": "tensor", "achieved": achieved, "peak": pk["tflops"],
             "unit": "TFLOP/s", "frac": achieved / pk["tflops"], "peak_source": pk["source"] + " (burst bf16)",
             "frac_of_sustained": (achieved / pk["tflops_sustained"]) if pk.get("tflops_sustained") else None,
             "avg_launch_ms": avg_route_ms, "bracketed_launch_ms": bracketed_ms,
