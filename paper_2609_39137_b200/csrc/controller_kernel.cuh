@@ -135,11 +135,23 @@ __device__ __forceinline__ void controller_layer(const CtrlParams& p, int layer,
     }
     sync();
 #pragma unroll 1
-    for (int stride = 512; stride >= 1; stride >>= 1) {
+    for (int stride = 512; stride >= 32; stride >>= 1) {
       // y[i + stride] is not written during this pass, so one barrier suffices
       for (int i = tid; i < stride; i += NT) sc->y[i] = __dadd_rn(sc->y[i], sc->y[i + stride]);
       sync();
     }
+    if (tid < 32) {
+      // strides 16 ... 1 stay inside the first warp: same additions, warp barriers instead of block barriers
+#pragma unroll
+      for (int stride = 16; stride >= 1; stride >>= 1) {
+        double v = 0.0;
+        if (tid < stride) v = __dadd_rn(sc->y[tid], sc->y[tid + stride]);
+        __syncwarp();
+        if (tid < stride) sc->y[tid] = v;
+        __syncwarp();
+      }
+    }
+    sync();
     const float mean = (float)__ddiv_rn(sc->y[0], (double)p.E);
 #pragma unroll
     for (int j = 0; j < PER; ++j) b[j] = __fsub_rn(b[j], mean);
