@@ -479,19 +479,21 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
     if (!ctx->qb_logits) return fail(ctx, MOE_ERR_STATE, "quantile controller: no routing step since the last update");
     if (c.qb_hist_bins > 0) {
       // footnote to Eq. 7: the target estimated from a per-expert margin histogram, one pass over the dump
-      const size_t smem = (size_t)c.qb_hist_bins * kQhCols * 4;
+      const size_t smem = qh_smem_bytes(c.qb_hist_bins);
       static bool attr_set[64] = {};
       if (!attr_set[ctx->device & 63]) {
         cudaError_t ae = cudaFuncSetAttribute(qb_margin_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              kQhMaxBins * kQhCols * 4);
+                                              (int)qh_smem_bytes(kQhMaxBins));
         if (ae != cudaSuccess) return cuda_fail(ctx, ae, "cudaFuncSetAttribute(qb_margin_hist_kernel)");
         attr_set[ctx->device & 63] = true;
       }
       const int groups = (c.num_experts + kQhCols - 1) / kQhCols;
-      const int per_sm = smem <= 32768 ? 6 : smem <= 65536 ? 3 : 1;
+      const int per_sm = smem <= 33000 ? 6 : smem <= 66000 ? 3 : 1;
       int splits = (per_sm * ctx->num_sms + groups - 1) / groups;
       const int max_splits = (ctx->qb_tokens + 127) / 128;
       if (splits > max_splits) splits = max_splits;
+      const int min_splits = (ctx->qb_tokens + kQhMaxRowsPerCta - 1) / kQhMaxRowsPerCta;   // 16-bit counters per CTA
+      if (splits < min_splits) splits = min_splits;
       if (splits < 1) splits = 1;
       for (int l = 0; l < c.num_layers; ++l) {
         QhParams q{};
@@ -503,7 +505,7 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
         q.hist = at<uint32_t>(ctx, ctx->lay.qb_hist);
         q.target = at<float>(ctx, ctx->lay.qb_target) + (size_t)l * c.num_experts;
         qb_margin_hist_kernel<<<dim3(groups, splits), kQhThreads, smem, st>>>(q);
-        qb_margin_hist_finish_kernel<<<(c.num_experts * 32 + 255) / 256, 256, 0, st>>>(q);
+        qb_margin_hist_finish_kernel<<<c.num_experts, kQhFinishThreads, 0, st>>>(q);
         ctx->launches += 2;
       }
       cudaError_t qe = cudaGetLastError();

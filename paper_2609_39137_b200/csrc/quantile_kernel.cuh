@@ -174,8 +174,11 @@ __global__ void qb_scan_kernel(QbParams p, int pass) {
 // the rule inside a bin are this library's choice).  One pass over the dump:
 //   bin k = floor((d + range) * inv_h) clamped to [0, B-1], d = sigmoid(z) - alpha
 //   (two rounded binary32 operations), B uniform bins over [-range, range);
-// the counts of a CTA's 16 experts are kept in shared memory ([bin][expert]) and
-// flushed with one global atomic per non-empty bin.  A second kernel (one warp
+// the counts of a CTA's 16 experts are kept in shared memory as 16-bit halves of
+// 32-bit words ([B/2][expert] words, so the 16 lanes of a row hit 16 banks; a CTA sees fewer than 65536 rows, so a
+// half cannot carry into its neighbour; half the footprint of 32-bit counters,
+// twice the resident CTAs) and flushed with one global atomic per non-empty bin,
+// consecutive lanes on consecutive bins of one expert (contiguous addresses).  A second kernel (one warp
 // per expert) finds the bin k* of the r-th smallest margin, r = m - floor(mK/E),
 // and interpolates in binary64: est = -range + (k* + ((r - below) - 0.5) / cnt) * h.
 // The counts are integers, so histograms of several ranks can be added before
@@ -184,7 +187,7 @@ __global__ void qb_scan_kernel(QbParams p, int pass) {
 constexpr int kQhCols = 16;        // experts per CTA
 constexpr int kQhThreads = 256;
 constexpr int kQhRowsInFlight = 8;
-constexpr int kQhMaxBins = 2048;   // 16 experts x 2048 bins x 4 bytes = 128 KB of shared memory
+constexpr int kQhMaxBins = 2048;   // 16 experts x 1024 words = 64 KB of shared memory
 
 struct QhParams {
   const float* logits;  // [m][E]
@@ -202,11 +205,14 @@ __device__ __forceinline__ int margin_bin(float d, float range, float inv_h, int
   return (fl >= (float)B) ? B - 1 : (int)fl;
 }
 
-// grid = (ceil(E / 16), row_splits); dynamic shared memory B * 16 * 4 bytes.  A warp covers two rows of 16
+__host__ __device__ inline size_t qh_smem_bytes(int B) { return (size_t)kQhCols * (B / 2) * 4; }
+constexpr int kQhMaxRowsPerCta = 65535;   // 16-bit counters
+
+// grid = (ceil(E / 16), row_splits); dynamic shared memory qh_smem_bytes(B).  A warp covers two rows of 16
 // experts (64 bytes each) per load; kQhRowsInFlight loads are issued before the first is used.
 __global__ void __launch_bounds__(kQhThreads) qb_margin_hist_kernel(QhParams p) {
-  extern __shared__ uint32_t hs[];   // [bin][col]
-  for (int i = threadIdx.x; i < p.B * kQhCols; i += kQhThreads) hs[i] = 0u;
+  extern __shared__ uint32_t hs[];   // [B / 2][col] words, two 16-bit counters each
+  for (int i = threadIdx.x; i < kQhCols * (p.B / 2); i += kQhThreads) hs[i] = 0u;
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = lane & (kQhCols - 1), sub = lane >> 4;
@@ -230,55 +236,71 @@ __global__ void __launch_bounds__(kQhThreads) qb_margin_hist_kernel(QhParams p) 
       const int i = i0 + u * kRowsPerIter;
       if (live && i < r1) {
         const float d = __fsub_rn(sigmoid_score(z[u]), a[u]);
-        atomicAdd(&hs[margin_bin(d, p.range, p.inv_h, p.B) * kQhCols + c], 1u);
+        const int bin = margin_bin(d, p.range, p.inv_h, p.B);
+        atomicAdd(&hs[(bin >> 1) * kQhCols + c], 1u << (16 * (bin & 1)));
       }
     }
   }
   __syncthreads();
   for (int i = threadIdx.x; i < p.B * kQhCols; i += kQhThreads) {
-    const int cc = blockIdx.x * kQhCols + (i & (kQhCols - 1));
-    const uint32_t cnt = hs[i];
-    if (cnt != 0u && cc < p.E) atomicAdd(&p.hist[(size_t)cc * p.B + (i >> 4)], cnt);
+    const int cl = i / p.B, bin = i - cl * p.B;       // B is a multiple of 32: a warp stays inside one expert
+    const int cc = blockIdx.x * kQhCols + cl;
+    const uint32_t cnt = (hs[(bin >> 1) * kQhCols + cl] >> (16 * (bin & 1))) & 0xffffu;
+    if (cnt != 0u && cc < p.E) atomicAdd(&p.hist[(size_t)cc * p.B + bin], cnt);
   }
 }
 
-// One warp per expert: lane l owns the bins [l * B/32, (l+1) * B/32) (B is a multiple of 32).
-__global__ void qb_margin_hist_finish_kernel(QhParams p) {
-  const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (j >= p.E) return;
+// One CTA of 256 threads per expert: thread t owns the bins [t * per, (t + 1) * per), per = ceil(B / 256); a block
+// scan of the threads' sums gives the count before each thread's range, and the thread whose range takes the
+// cumulative count to the rank or beyond walks its bins and interpolates.  Every thread clears its bins (ready
+// for the next update).
+constexpr int kQhFinishThreads = 256;
+
+__global__ void __launch_bounds__(kQhFinishThreads) qb_margin_hist_finish_kernel(QhParams p) {
+  __shared__ uint32_t warp_tot[kQhFinishThreads / 32];
+  const int j = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t* hj = p.hist + (size_t)j * p.B;
-  const int per = p.B / 32;
+  const int per = (p.B + kQhFinishThreads - 1) / kQhFinishThreads;    // <= 8 for B <= 2048
+  const int b0 = tid * per;
+  uint32_t c[8];
   uint32_t mine = 0;
-  for (int t = 0; t < per; ++t) mine += hj[lane * per + t];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    c[t] = (t < per && b0 + t < p.B) ? hj[b0 + t] : 0u;
+    mine += c[t];
+  }
+#pragma unroll
+  for (int t = 0; t < 8; ++t)
+    if (t < per && b0 + t < p.B) hj[b0 + t] = 0u;
   uint32_t incl = mine;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
     const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
     if (lane >= d) incl += o;
   }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  uint32_t before = incl - mine;                          // count of the bins before this thread's range
+  for (int w = 0; w < warp; ++w) before += warp_tot[w];
   long long r = (long long)p.m - ((long long)p.m * p.K) / p.E;
   if (r < 1) r = 1;
   if (r > p.m) r = p.m;
   const uint32_t rank = (uint32_t)r;
-  const uint32_t excl = incl - mine;
-  if (rank > excl && rank <= incl) {           // exactly one lane: the counts of an expert sum to m >= rank
-    uint32_t run = excl;
-    for (int t = 0; t < per; ++t) {
-      const uint32_t cnt = hj[lane * per + t];
-      if (rank <= run + cnt) {
-        const int kstar = lane * per + t;
+  if (rank > before && rank <= before + mine) {           // exactly one thread: the counts of an expert sum to m >= rank
+    uint32_t run = before;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if (rank > run && rank <= run + c[t]) {
+        const int kstar = b0 + t;
         const double h = __ddiv_rn(__dmul_rn(2.0, (double)p.range), (double)p.B);
-        const double inside = __ddiv_rn(__dsub_rn((double)(rank - run), 0.5), (double)cnt);
+        const double inside = __ddiv_rn(__dsub_rn((double)(rank - run), 0.5), (double)c[t]);
         const double est = __dadd_rn(-(double)p.range, __dmul_rn(__dadd_rn((double)kstar, inside), h));
         p.target[j] = -(float)est;
-        break;
       }
-      run += cnt;
+      run += c[t];
     }
   }
-  __syncwarp();
-  for (int t = 0; t < per; ++t) hj[lane * per + t] = 0u;   // ready for the next update
 }
 
 }  // namespace moe
