@@ -28,7 +28,7 @@ def test_small_parity_cases_pass_on_the_debug_build():
     lib = build.build(debug=True)
     env = dict(os.environ, MOE_ROUTE_LIB=lib)
     select = ("test_route_matches_oracle or test_route_edge_shapes or chunk_split_scheduling or random_shapes "
-              "or gives_up or exact_ties or canary or one_launch")
+              "or gives_up or exact_ties or canary or one_launch or non_finite")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-v", "-m", "gpu", "-p", "no:cacheprovider",
                         os.path.join("tests", "test_gpu_parity.py"), os.path.join("tests", "test_debug_build.py"),
                         "-k", select], env=env, cwd=ROOT, capture_output=True, text=True, timeout=1200)

@@ -118,6 +118,33 @@ def test_route_exact_ties_pick_lowest_index():
     full_check(res, K)
 
 
+@pytest.mark.parametrize("chunk_split", [1, 2])
+def test_non_finite_hidden_states_do_not_disturb_other_tokens(chunk_split):
+    # the paper says nothing about NaN / Inf activations; the library's promise is only that they cannot fault and
+    # cannot leak into other tokens: rows with finite inputs route exactly as without the bad rows, every index
+    # written for a bad row is a valid expert or the "no expert" marker, and the loads count only valid experts
+    T, H, E, K = 400, 128, 768, 10
+    g = torch.Generator(device="cuda").manual_seed(3)
+    x = torch.randn(1, T, H, device="cuda", generator=g).to(torch.bfloat16)
+    w = (torch.randn(1, E, H, device="cuda", generator=g) / 11).to(torch.bfloat16)
+    clean = route_once(T, H, E, K, x=x, w=w, chunk_split=chunk_split)
+    bad_rows = [5, 130, 131, 399]
+    xb = x.clone()
+    xb[0, 5, 7] = float("nan")
+    xb[0, 130, :] = float("inf")
+    xb[0, 131, 0] = float("-inf")
+    xb[0, 399, 100] = float("nan")
+    res = route_once(T, H, E, K, x=xb, w=w, chunk_split=chunk_split)
+    assert res["r"].poll(raise_on_error=False) == binding.MOE_OK
+    good = np.setdiff1d(np.arange(T), bad_rows)
+    np.testing.assert_array_equal(res["idx"][0][good], clean["idx"][0][good])
+    np.testing.assert_array_equal(bits(res["gate"][0][good]), bits(clean["gate"][0][good]))
+    bad_idx = res["idx"][0][bad_rows]
+    assert np.all(((bad_idx >= 0) & (bad_idx < E)) | (bad_idx == 0x7fffffff))
+    valid = res["idx"][0][(res["idx"][0] >= 0) & (res["idx"][0] < E)]
+    np.testing.assert_array_equal(res["loads"][0], np.bincount(valid, minlength=E))
+
+
 def test_route_is_deterministic_and_accumulates_microbatches():
     T, H, E, K, L = 700, 256, 768, 10, 2
     a = route_once(T, H, E, K, L, seed=5)
