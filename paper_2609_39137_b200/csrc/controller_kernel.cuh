@@ -15,6 +15,8 @@
 #include <limits.h>
 #include <stdint.h>
 
+#include "route_math.cuh"
+
 namespace moe {
 
 constexpr int kCtrlThreads = 1024;
@@ -207,6 +209,7 @@ struct DiagParams {
 };
 
 __global__ void __launch_bounds__(kCtrlThreads) diagnostics_kernel(const DiagParams p) {
+  chained_launch_enter();
   __shared__ unsigned int hist[256];
   __shared__ unsigned int sel_prefix, sel_rank;
   __shared__ long long red_a[32], red_b[32];
@@ -297,6 +300,7 @@ constexpr int kEntropySlices = 64;
 constexpr int kEntropyThreads = 256;
 
 __global__ void __launch_bounds__(kEntropyThreads) gate_entropy_kernel(const float* gate, int T, int K, double* part) {
+  chained_launch_enter();
   __shared__ double y[kEntropyThreads];
   const int layer = blockIdx.y, slice = blockIdx.x, i = threadIdx.x;
   const int per = (T + kEntropySlices - 1) / kEntropySlices;
@@ -321,6 +325,7 @@ __global__ void __launch_bounds__(kEntropyThreads) gate_entropy_kernel(const flo
 }
 
 __global__ void gate_entropy_finish_kernel(const double* part, int T, float* out) {
+  chained_launch_enter();
   const int layer = blockIdx.x;
   if (threadIdx.x == 0) {
     double s = 0.0;
@@ -333,6 +338,7 @@ __global__ void gate_entropy_finish_kernel(const double* part, int T, float* out
 // routing kernel's tensor maps describe).  64 x 64 tiles through shared memory; grid (ceil(E/64), ceil(H/64), L),
 // 256 threads; reads and writes are 128-byte rows.
 __global__ void __launch_bounds__(256) transpose_w_kernel(const uint16_t* in, uint16_t* out, int H, int E) {
+  chained_launch_enter();
   __shared__ uint16_t tile[64][66];
   const int layer = blockIdx.z, e0 = blockIdx.x * 64, h0 = blockIdx.y * 64;
   const uint16_t* src = in + (size_t)layer * H * E;
@@ -351,6 +357,7 @@ __global__ void __launch_bounds__(256) transpose_w_kernel(const uint16_t* in, ui
 
 // loads_acc[i] += add[i]
 __global__ void loads_add_kernel(int* acc, const int* add, int n) {
+  chained_launch_enter();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) acc[i] += add[i];
 }

@@ -211,6 +211,23 @@ int encode_map(moe_route_ctx* ctx, CUtensorMap* out, const void* base, uint64_t 
   return MOE_OK;
 }
 
+// Launch with programmatic stream serialisation: the kernel's launch latency and prologue overlap the tail of the
+// kernel queued before it; every kernel launched this way starts with chained_launch_enter().
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &attr;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
+}
+
 template <int KL>
 int launch_route(moe_route_ctx* ctx, const RouteParams& rp, int grid, cudaStream_t st) {
   static bool attr_set[64] = {};
@@ -247,7 +264,7 @@ int route_device(moe_route_ctx* ctx, const void* x, const void* w, int32_t T, in
     if (reinterpret_cast<uintptr_t>(w) & 1) return fail(ctx, MOE_ERR_INVALID_ARG, "w must be 2-byte aligned");
     uint16_t* wt = at<uint16_t>(ctx, ctx->lay.w_t);
     const dim3 tg((c.num_experts + 63) / 64, (c.hidden + 63) / 64, c.num_layers);
-    transpose_w_kernel<<<tg, 256, 0, st>>>(static_cast<const uint16_t*>(w), wt, c.hidden, c.num_experts);
+    launch_chained(transpose_w_kernel, tg, dim3(256), 0, st, static_cast<const uint16_t*>(w), wt, c.hidden, c.num_experts);
     cudaError_t te = cudaGetLastError();
     if (te != cudaSuccess) return cuda_fail(ctx, te, "transpose_w_kernel launch");
     ctx->launches += 1;
@@ -504,8 +521,8 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
         q.inv_h = (float)c.qb_hist_bins / (2.0f * c.qb_hist_range);
         q.hist = at<uint32_t>(ctx, ctx->lay.qb_hist);
         q.target = at<float>(ctx, ctx->lay.qb_target) + (size_t)l * c.num_experts;
-        qb_margin_hist_kernel<<<dim3(groups, splits), kQhThreads, smem, st>>>(q);
-        qb_margin_hist_finish_kernel<<<c.num_experts, kQhFinishThreads, 0, st>>>(q);
+        launch_chained(qb_margin_hist_kernel, dim3(groups, splits), dim3(kQhThreads), smem, st, q);
+        launch_chained(qb_margin_hist_finish_kernel, dim3(c.num_experts), dim3(kQhFinishThreads), 0, st, q);
         ctx->launches += 2;
       }
       cudaError_t qe = cudaGetLastError();
@@ -528,10 +545,10 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
       q.rank = at<uint32_t>(ctx, ctx->lay.qb_rank);
       q.target = at<float>(ctx, ctx->lay.qb_target) + (size_t)l * c.num_experts;
       q.keys = at<uint32_t>(ctx, ctx->lay.qb_keys);
-      qb_init_kernel<<<64, 256, 0, st>>>(q);
+      launch_chained(qb_init_kernel, dim3(64), dim3(256), 0, st, q);
       for (int pass = 0; pass < 4; ++pass) {
-        qb_hist_kernel<<<dim3(col_groups, splits), kQbThreads, 0, st>>>(q, pass);
-        qb_scan_kernel<<<(c.num_experts * 32 + 255) / 256, 256, 0, st>>>(q, pass);
+        launch_chained(qb_hist_kernel, dim3(col_groups, splits), dim3(kQbThreads), 0, st, q, pass);
+        launch_chained(qb_scan_kernel, dim3((c.num_experts * 32 + 255) / 256), dim3(256), 0, st, q, pass);
       }
       ctx->launches += 9;
     }
@@ -615,7 +632,7 @@ int moe_load_diagnostics(moe_route_ctx* ctx, float* diag, void* cuda_stream) {
   d.bias = at<float>(ctx, ctx->lay.bias);
   d.bias_prev = at<float>(ctx, ctx->lay.bias_prev);
   d.out = diag;
-  diagnostics_kernel<<<d.L, kCtrlThreads, 0, st>>>(d);
+  launch_chained(diagnostics_kernel, dim3(d.L), dim3(kCtrlThreads), 0, st, d);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "diagnostics_kernel launch");
   ctx->launches += 1;
@@ -629,11 +646,11 @@ int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tok
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   ctx->last_stream = st;
   double* part = at<double>(ctx, ctx->lay.ent_part);
-  gate_entropy_kernel<<<dim3(kEntropySlices, ctx->cfg.num_layers), kEntropyThreads, 0, st>>>(topk_gate, num_tokens,
-                                                                                           ctx->cfg.top_k, part);
+  launch_chained(gate_entropy_kernel, dim3(kEntropySlices, ctx->cfg.num_layers), dim3(kEntropyThreads), 0, st, topk_gate,
+                 num_tokens, ctx->cfg.top_k, part);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "gate_entropy_kernel launch");
-  gate_entropy_finish_kernel<<<ctx->cfg.num_layers, 32, 0, st>>>(part, num_tokens, entropy);
+  launch_chained(gate_entropy_finish_kernel, dim3(ctx->cfg.num_layers), dim3(32), 0, st, part, num_tokens, entropy);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "gate_entropy_finish_kernel launch");
   ctx->launches += 2;
@@ -658,16 +675,16 @@ int moe_score_stats(moe_route_ctx* ctx, const float* logits, int32_t num_tokens,
   p.aux_part = at<double>(ctx, ctx->lay.stat_aux);
   p.loads = loads; p.h_biased = entropy_biased; p.h_softmax = entropy_softmax; p.mean_prob = mean_prob; p.aux = aux;
   const dim3 grid(p.C, p.L);
-  if (p.E <= 256) score_stats_kernel<8><<<grid, kStatThreads, 0, st>>>(p);
-  else if (p.E <= 768) score_stats_kernel<24><<<grid, kStatThreads, 0, st>>>(p);
-  else score_stats_kernel<32><<<grid, kStatThreads, 0, st>>>(p);
+  if (p.E <= 256) launch_chained(score_stats_kernel<8>, grid, dim3(kStatThreads), 0, st, p);
+  else if (p.E <= 768) launch_chained(score_stats_kernel<24>, grid, dim3(kStatThreads), 0, st, p);
+  else launch_chained(score_stats_kernel<32>, grid, dim3(kStatThreads), 0, st, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_kernel launch");
   const int groups = (p.E + kStatFinExperts - 1) / kStatFinExperts;
-  score_stats_finish_kernel<<<dim3(groups, p.L), 1024, 0, st>>>(p);
+  launch_chained(score_stats_finish_kernel, dim3(groups, p.L), dim3(1024), 0, st, p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_finish_kernel launch");
-  score_stats_scalar_kernel<<<p.L, 32, 0, st>>>(p, groups);
+  launch_chained(score_stats_scalar_kernel, dim3(p.L), dim3(32), 0, st, p, groups);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_scalar_kernel launch");
   ctx->launches += 3;
@@ -695,7 +712,7 @@ int moe_loads_add(moe_route_ctx* ctx, const int32_t* loads, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   ctx->last_stream = st;
   const int n = ctx->cfg.num_layers * ctx->cfg.num_experts;
-  loads_add_kernel<<<(n + 255) / 256, 256, 0, st>>>(at<int>(ctx, ctx->lay.loads_acc), loads, n);
+  launch_chained(loads_add_kernel, dim3((n + 255) / 256), dim3(256), 0, st, at<int>(ctx, ctx->lay.loads_acc), loads, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "loads_add_kernel launch");
   ctx->launches += 1;
@@ -878,15 +895,15 @@ int moe_quantile_target_static(const float* logits, const float* alpha, int32_t 
   q.target = target_out;
   // the array keeps whatever the previous call left: the init kernel clears the histogram and
   // resets prefix and rank before anything is counted
-  qb_init_kernel<<<64, 256, 0, st>>>(q);
+  launch_chained(qb_init_kernel, dim3(64), dim3(256), 0, st, q);
   const int col_groups = (num_experts + kQbCols - 1) / kQbCols;
   int splits = (6 * g_static_sms[dev] + col_groups - 1) / col_groups;
   const int max_splits = (num_tokens + 63) / 64;
   if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;
   for (int pass = 0; pass < 4; ++pass) {
-    qb_hist_kernel<<<dim3(col_groups, splits), kQbThreads, 0, st>>>(q, pass);
-    qb_scan_kernel<<<(num_experts * 32 + 255) / 256, 256, 0, st>>>(q, pass);
+    launch_chained(qb_hist_kernel, dim3(col_groups, splits), dim3(kQbThreads), 0, st, q, pass);
+    launch_chained(qb_scan_kernel, dim3((num_experts * 32 + 255) / 256), dim3(256), 0, st, q, pass);
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -52,6 +52,7 @@ __device__ __forceinline__ float margin_from_key(uint32_t k) {
 }
 
 __global__ void qb_init_kernel(QbParams p) {
+  chained_launch_enter();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j < p.E) {
     long long r = (long long)p.m - ((long long)p.m * p.K) / p.E;
@@ -65,6 +66,7 @@ __global__ void qb_init_kernel(QbParams p) {
 
 // pass = 0..3, most significant byte first.  grid = (ceil(E/32), row_splits)
 __global__ void __launch_bounds__(kQbThreads) qb_hist_kernel(QbParams p, int pass) {
+  chained_launch_enter();
   __shared__ uint32_t h[256 * kQbCols];  // [bin][col]: lanes hit distinct banks
   for (int i = threadIdx.x; i < 256 * kQbCols; i += kQbThreads) h[i] = 0u;
   __syncthreads();
@@ -128,6 +130,7 @@ __global__ void __launch_bounds__(kQbThreads) qb_hist_kernel(QbParams p, int pas
 // One warp per expert: find the bin holding the remaining rank, fix that
 // digit, clear the histogram; after the last pass emit Q_j = -margin.
 __global__ void qb_scan_kernel(QbParams p, int pass) {
+  chained_launch_enter();
   const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (j >= p.E) return;
@@ -211,6 +214,7 @@ constexpr int kQhMaxRowsPerCta = 65535;   // 16-bit counters
 // grid = (ceil(E / 16), row_splits); dynamic shared memory qh_smem_bytes(B).  A warp covers two rows of 16
 // experts (64 bytes each) per load; kQhRowsInFlight loads are issued before the first is used.
 __global__ void __launch_bounds__(kQhThreads) qb_margin_hist_kernel(QhParams p) {
+  chained_launch_enter();
   extern __shared__ uint32_t hs[];   // [B / 2][col] words, two 16-bit counters each
   for (int i = threadIdx.x; i < kQhCols * (p.B / 2); i += kQhThreads) hs[i] = 0u;
   __syncthreads();
@@ -257,6 +261,7 @@ __global__ void __launch_bounds__(kQhThreads) qb_margin_hist_kernel(QhParams p) 
 constexpr int kQhFinishThreads = 256;
 
 __global__ void __launch_bounds__(kQhFinishThreads) qb_margin_hist_finish_kernel(QhParams p) {
+  chained_launch_enter();
   __shared__ uint32_t warp_tot[kQhFinishThreads / 32];
   const int j = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

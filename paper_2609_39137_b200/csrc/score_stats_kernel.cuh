@@ -78,6 +78,7 @@ __device__ __forceinline__ float warp_max(float v) {
 // NPL = experts per lane (E <= 32 * NPL).  grid = (C, L)
 template <int NPL>
 __global__ void __launch_bounds__(kStatThreads, 4) score_stats_kernel(StatParams p) {
+  chained_launch_enter();
   // per-warp accumulators of the softmax probabilities and the layer's bias live in shared memory so that
   // a thread's registers hold little more than its NPL logits of the current row (4 CTAs per SM)
   __shared__ float sP[kStatWarps][32 * NPL];
@@ -158,6 +159,7 @@ constexpr int kStatFinSlices = 16;
 constexpr int kStatMaxGroups = 16;   // 1024 experts / 64
 
 __global__ void __launch_bounds__(1024) score_stats_finish_kernel(StatParams p) {
+  chained_launch_enter();
   __shared__ double y[kStatFinSlices][kStatFinExperts];
   const int layer = blockIdx.y, group = blockIdx.x;
   const int el = threadIdx.x % kStatFinExperts, sl = threadIdx.x / kStatFinExperts;
@@ -189,6 +191,7 @@ __global__ void __launch_bounds__(1024) score_stats_finish_kernel(StatParams p) 
 
 // Third step, one warp per layer: the groups' aux shares and the per-CTA entropy sums, added in index order.
 __global__ void score_stats_scalar_kernel(StatParams p, int groups) {
+  chained_launch_enter();
   const int layer = blockIdx.x, lane = threadIdx.x;
   double hb = 0.0, hs = 0.0;
   for (int c = lane; c < p.C; c += 32) {
