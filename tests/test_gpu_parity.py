@@ -409,10 +409,11 @@ def test_quantile_target_count_property_on_gpu_result():
         r.controller_update()
 
 
-def test_host_buffer_step_matches_device_step():
+@pytest.mark.parametrize("chunk_split", [1, 2])
+def test_host_buffer_step_matches_device_step(chunk_split):
     T, H, E, K, L = 900, 256, 768, 10, 2
-    res = route_once(T, H, E, K, L, seed=9)
-    r = binding.Router(L, E, K, H, T, host_staging=True)
+    res = route_once(T, H, E, K, L, seed=9, chunk_split=chunk_split)
+    r = binding.Router(L, E, K, H, T, host_staging=True, chunk_split=chunk_split)
     xh, wh = res["x"].cpu().pin_memory(), res["w"].cpu().pin_memory()
     ih = torch.empty(L, T, K, dtype=torch.int32).pin_memory()
     gh = torch.empty(L, T, K, dtype=torch.float32).pin_memory()
@@ -564,15 +565,17 @@ def test_expert_contiguous_weight_layout(T, H, E, K, L):
     np.testing.assert_array_equal(ih.numpy(), res["idx"])
 
 
-def test_step_replays_from_a_cuda_graph():
-    # routing + controller update captured once into a CUDA graph (both launches use programmatic stream
-    # serialisation) and replayed: state and outputs evolve exactly as with eager launches
+@pytest.mark.parametrize("chunk_split", [1, 2])
+def test_step_replays_from_a_cuda_graph(chunk_split):
+    # routing (+ the merge kernel under chunk-split scheduling) + controller update captured once into a CUDA graph
+    # (all launches use programmatic stream serialisation) and replayed: state and outputs evolve exactly as with
+    # eager launches
     T, H, E, K, L = 640, 256, 768, 10, 2
     g = torch.Generator(device="cuda").manual_seed(77)
     x = torch.randn(L, T, H, device="cuda", generator=g).to(torch.bfloat16)
     w = (torch.randn(L, E, H, device="cuda", generator=g) / 16).to(torch.bfloat16)
-    eager = binding.Router(L, E, K, H, T)
-    graphed = binding.Router(L, E, K, H, T)
+    eager = binding.Router(L, E, K, H, T, chunk_split=chunk_split)
+    graphed = binding.Router(L, E, K, H, T, chunk_split=chunk_split)
     idx_e = torch.empty(L, T, K, dtype=torch.int32, device="cuda")
     gate_e = torch.empty(L, T, K, device="cuda")
     idx_g, gate_g = torch.empty_like(idx_e), torch.empty_like(gate_e)
