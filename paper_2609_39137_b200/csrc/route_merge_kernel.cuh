@@ -16,8 +16,8 @@
 //
 // Memory-bound: per token it reads num_chunks * cand_len * 8 bytes and writes
 // 8 K (+4) bytes.  A warp takes 32 consecutive tokens: their lists are one
-// contiguous block, which the lanes fetch with coalesced loads (batches of
-// independent loads in flight) into the warp's part of shared memory, one row
+// contiguous block, which the lanes fetch with coalesced asynchronous copies
+// (all in flight at once) into the warp's part of shared memory, one row
 // per token with an odd row stride (conflict-free both for the staging and for
 // the lanes reading different entries of their own rows); then each lane
 // merges its own token from there and stores its outputs.  A CTA walks tokens
@@ -34,7 +34,6 @@ namespace moe {
 constexpr int kMergeThreads = 256;
 constexpr int kMergeMaxChunks = 4;     // 1024 experts / 256 per chunk
 constexpr int kMergeMaxK = 16;
-constexpr int kMergeBatch = 8;         // independent loads in flight per thread
 
 struct MergeParams {
   int T, E, K, num_chunks, cand_len;
@@ -53,7 +52,7 @@ __host__ __device__ inline size_t merge_smem_bytes(int n_all) {
 }
 
 // grid = (slices, L); dynamic shared memory merge_smem_bytes(num_chunks * cand_len)
-__global__ void __launch_bounds__(kMergeThreads) route_merge_kernel(const MergeParams p) {
+__global__ void __launch_bounds__(kMergeThreads, 3) route_merge_kernel(const MergeParams p) {
   extern __shared__ float2 lists_s[];                       // [entry][thread]
   __shared__ float bias_s[1024];
   __shared__ int hist_s[1024];
@@ -83,19 +82,16 @@ __global__ void __launch_bounds__(kMergeThreads) route_merge_kernel(const MergeP
     int r = 0, n = lane;                                   // element lane + 32 j as (row, entry)
     while (n >= n_all) { n -= n_all; r += 1; }
     const int dr = 32 / n_all, dn = 32 - dr * n_all;       // advancing the element by 32
+    // asynchronous 8-byte copies global -> shared, all of the group's entries in flight at once (no registers
+    // are held for them); consecutive lanes, consecutive entries
 #pragma unroll 1
-    for (int i0 = lane; i0 < total + lane; i0 += 32 * kMergeBatch) {
-      float2 t[kMergeBatch];
-#pragma unroll
-      for (int u = 0; u < kMergeBatch; ++u)
-        t[u] = (i0 + 32 * u < total) ? __ldg(src + i0 + 32 * u) : make_float2(0.0f, 0.0f);
-#pragma unroll
-      for (int u = 0; u < kMergeBatch; ++u) {
-        if (i0 + 32 * u < total) warp_s[r * stride + n] = t[u];
-        r += dr; n += dn;
-        if (n >= n_all) { n -= n_all; r += 1; }
-      }
+    for (int i = lane; i < total; i += 32) {
+      const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(warp_s + r * stride + n));
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src + i) : "memory");
+      r += dr; n += dn;
+      if (n >= n_all) { n -= n_all; r += 1; }
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");
     __syncwarp();
     const int tok = tok0 + lane;
     if (lane < rows) {
