@@ -27,7 +27,7 @@ constexpr size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign;
 
 struct Layout {
   size_t status, bias, e_prev, bias_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
-  size_t qb_target, qb_hist, qb_prefix, qb_rank, qb_keys;
+  size_t qb_target, qb_hist, qb_prefix, qb_rank, qb_keys, qb_match, qb_fill, qb_list;
   size_t state_end;  // everything before this is cleared at init
   size_t stat_P, stat_H, stat_aux, ent_part;   // per-CTA partial sums of moe_score_stats (written before they are read)
   size_t stage_x, stage_w, stage_idx, stage_gate;
@@ -87,8 +87,12 @@ Layout make_layout(const moe_route_config& c) {
     l.qb_rank = take((size_t)c.num_experts * 4);
   }
   l.state_end = o;
-  if (c.controller == MOE_CTRL_QUANTILE && c.qb_hist_bins == 0)
+  if (c.controller == MOE_CTRL_QUANTILE && c.qb_hist_bins == 0) {
     l.qb_keys = take((size_t)c.max_tokens * c.num_experts * 4);
+    l.qb_match = take((size_t)c.num_experts * 4);
+    l.qb_fill = take((size_t)c.num_experts * 4);
+    l.qb_list = take((size_t)c.num_experts * kQbListCap * 2);
+  }
   {
     const size_t LC = (size_t)c.num_layers * stat_ctas_per_layer(c.num_layers);
     l.stat_P = take(LC * c.num_experts * 4);
@@ -545,12 +549,19 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
       q.rank = at<uint32_t>(ctx, ctx->lay.qb_rank);
       q.target = at<float>(ctx, ctx->lay.qb_target) + (size_t)l * c.num_experts;
       q.keys = at<uint32_t>(ctx, ctx->lay.qb_keys);
+      q.match = at<uint32_t>(ctx, ctx->lay.qb_match);
+      q.fill = at<uint32_t>(ctx, ctx->lay.qb_fill);
+      q.list = at<uint16_t>(ctx, ctx->lay.qb_list);
       launch_chained(qb_init_kernel, dim3(64), dim3(256), 0, st, q);
-      for (int pass = 0; pass < 4; ++pass) {
+      for (int pass = 0; pass < 2; ++pass) {
         launch_chained(qb_hist_kernel, dim3(col_groups, splits), dim3(kQbThreads), 0, st, q, pass);
         launch_chained(qb_scan_kernel, dim3((c.num_experts * 32 + 255) / 256), dim3(256), 0, st, q, pass);
       }
-      ctx->launches += 9;
+      // the last two digits: gather the keys that share the 16-bit prefix, select among them
+      launch_chained(qb_gather_kernel, dim3(col_groups, splits), dim3(kQbThreads), 0, st, q);
+      launch_chained(qb_select_kernel, dim3((c.num_experts + kQbSelectWarps - 1) / kQbSelectWarps),
+                     dim3(kQbSelectWarps * 32), 0, st, q);
+      ctx->launches += 7;
     }
     {
       cudaError_t qe = cudaGetLastError();

@@ -15,7 +15,14 @@
 // stream those 4 bytes back instead of recomputing the score, which makes them
 // memory-bound instead of instruction-bound.
 //
-// Scratch per context: hist [E][256] u32, prefix [E] u32, rank [E] u32, keys [max_tokens][E] u32.
+// Contexts with the key scratch replace the last two digit passes by a gather:
+// after two passes the keys sharing the answer's 16-bit prefix are few (their
+// number is the count of the bin the second scan chose); one more stream over
+// the keys appends them to a per-expert list, and a warp per expert selects the
+// answer among them (two 8-bit digits in shared memory).
+//
+// Scratch per context: hist [E][256] u32, prefix [E] u32, rank [E] u32, keys [max_tokens][E] u32,
+// match [E] u32, fill [E] u32, list [E][1024] u16.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -37,7 +44,13 @@ struct QbParams {
   uint32_t* rank;       // [E] remaining 1-based rank inside the matching set
   float* target;        // [E] out: Q_j
   uint32_t* keys;       // [m][E] scratch or null: pass 0 stores every margin's key, later passes read it back
+  // gather form of the last two digits (contexts with a key scratch): after two passes the keys that share the
+  // 16-bit prefix of the answer are few; they are gathered per expert and the answer is selected among them
+  uint32_t* match;      // [E] number of keys sharing the prefix (the count of the bin chosen by the second scan)
+  uint32_t* fill;       // [E] entries gathered so far
+  uint16_t* list;       // [E][kQbListCap] low 16 bits of the gathered keys
 };
+constexpr int kQbListCap = 1024;
 
 // Monotone map float -> uint32 (a < b as floats  <=>  key(a) < key(b)); -0 is
 // canonicalised to +0 first so equal values get equal keys.
@@ -148,12 +161,12 @@ __global__ void qb_scan_kernel(QbParams p, int pass) {
   const uint32_t rank = p.rank[j];
   const uint32_t excl = incl - mine;
   const bool holder = (rank > excl) && (rank <= incl);   // exactly one lane when 1 <= rank <= total
-  uint32_t bin = 0, below = 0;
+  uint32_t bin = 0, below = 0, count = 0;
   if (holder) {
     uint32_t run = excl;
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
-      if (rank > run && rank <= run + c[t]) { bin = lane * 8 + t; below = run; }
+      if (rank > run && rank <= run + c[t]) { bin = lane * 8 + t; below = run; count = c[t]; }
       run += c[t];
     }
   }
@@ -161,6 +174,7 @@ __global__ void qb_scan_kernel(QbParams p, int pass) {
   const int src = who ? (__ffs(who) - 1) : 0;
   bin = __shfl_sync(0xffffffffu, bin, src);
   below = __shfl_sync(0xffffffffu, below, src);
+  count = __shfl_sync(0xffffffffu, count, src);
 #pragma unroll
   for (int t = 0; t < 8; ++t) hj[lane * 8 + t] = 0u;
   if (lane == 0) {
@@ -168,7 +182,109 @@ __global__ void qb_scan_kernel(QbParams p, int pass) {
     p.prefix[j] = pre;
     p.rank[j] = rank - below;
     if (pass == 3) p.target[j] = -margin_from_key(pre);
+    if (pass == 1 && p.match != nullptr) { p.match[j] = count; p.fill[j] = 0u; }
   }
+}
+
+// Gather (after two digit passes): one more stream over the stored keys; a key that shares the 16-bit prefix of
+// its expert's answer is appended to that expert's list (its low 16 bits).  Experts whose matching set is larger
+// than the list (long runs of equal margins) are left to the selection kernel, which then reads their keys itself.
+// grid and row split as for qb_hist_kernel.
+__global__ void __launch_bounds__(kQbThreads) qb_gather_kernel(QbParams p) {
+  chained_launch_enter();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int col = blockIdx.x * kQbCols + lane;
+  const bool live = col < p.E && p.match[col] <= (uint32_t)kQbListCap;
+  const uint32_t pre = live ? p.prefix[col] : 0u;
+  const int rows_per = (p.m + gridDim.y - 1) / gridDim.y;
+  const int r0 = blockIdx.y * rows_per;
+  const int r1 = min(p.m, r0 + rows_per);
+  constexpr int kWarps = kQbThreads / 32;
+  for (int i0 = r0 + warp; i0 < r1; i0 += kWarps * kQbRowsInFlight) {
+    uint32_t key[kQbRowsInFlight];
+#pragma unroll
+    for (int u = 0; u < kQbRowsInFlight; ++u) {
+      const int i = i0 + u * kWarps;
+      key[u] = (live && i < r1) ? __ldg(p.keys + (size_t)i * p.E + col) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < kQbRowsInFlight; ++u) {
+      const int i = i0 + u * kWarps;
+      if (live && i < r1 && ((key[u] ^ pre) >> 16) == 0u) {
+        const uint32_t pos = atomicAdd(&p.fill[col], 1u);
+        if (pos < (uint32_t)kQbListCap) p.list[(size_t)col * kQbListCap + pos] = (uint16_t)(key[u] & 0xffffu);
+      }
+    }
+  }
+}
+
+// Selection among the gathered keys: one warp per expert.  Two 8-bit digits over the low 16 bits, each a
+// warp-private shared-memory histogram followed by the same scan as qb_scan_kernel.  An expert whose matching
+// set did not fit the list walks its own column of the key scratch instead (strided reads: slow, but only long
+// runs of equal margins get there).  Emits Q_j = -margin.
+constexpr int kQbSelectWarps = 4;
+
+__global__ void __launch_bounds__(kQbSelectWarps * 32) qb_select_kernel(QbParams p) {
+  chained_launch_enter();
+  __shared__ uint32_t hs[kQbSelectWarps][256];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int j = blockIdx.x * kQbSelectWarps + warp;
+  if (j >= p.E) return;
+  uint32_t* h = hs[warp];
+  const uint32_t n_match = p.match[j];
+  const bool listed = n_match <= (uint32_t)kQbListCap;
+  const uint32_t n = listed ? n_match : (uint32_t)p.m;
+  uint32_t pre = p.prefix[j];          // top 16 bits fixed
+  uint32_t rank = p.rank[j];           // 1-based rank inside the matching set
+  const uint16_t* lst = p.list + (size_t)j * kQbListCap;
+  auto value = [&](uint32_t i, bool& match) -> uint32_t {
+    // low 16 bits of candidate i and whether it belongs to the matching set at all
+    if (listed) { match = true; return (uint32_t)lst[i]; }
+    const uint32_t key = __ldg(p.keys + (size_t)i * p.E + j);
+    match = ((key ^ pre) >> 16) == 0u;
+    return key & 0xffffu;
+  };
+#pragma unroll 1
+  for (int digit = 0; digit < 2; ++digit) {
+    const int shift = 8 - 8 * digit;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) h[lane * 8 + t] = 0u;
+    __syncwarp();
+    for (uint32_t i = lane; i < n; i += 32) {
+      bool match;
+      const uint32_t v = value(i, match);
+      if (match && (digit == 0 || ((v ^ pre) & 0xff00u) == 0u)) atomicAdd(&h[(v >> shift) & 255u], 1u);
+    }
+    __syncwarp();
+    uint32_t c[8], mine = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { c[t] = h[lane * 8 + t]; mine += c[t]; }
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
+    }
+    const uint32_t excl = incl - mine;
+    const bool holder = (rank > excl) && (rank <= incl);
+    uint32_t bin = 0, below = 0;
+    if (holder) {
+      uint32_t run = excl;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        if (rank > run && rank <= run + c[t]) { bin = lane * 8 + t; below = run; }
+        run += c[t];
+      }
+    }
+    const uint32_t who = __ballot_sync(0xffffffffu, holder);
+    const int src = who ? (__ffs(who) - 1) : 0;
+    bin = __shfl_sync(0xffffffffu, bin, src);
+    below = __shfl_sync(0xffffffffu, below, src);
+    pre |= bin << shift;
+    rank -= below;
+    __syncwarp();
+  }
+  if (lane == 0) p.target[j] = -margin_from_key(pre);
 }
 
 // ---------------------------------------------------------------------------

@@ -385,6 +385,27 @@ def test_closed_loop_drifting_deep_stack_opens_the_derivative_gate():
     assert max(h[2] for h in hist[1:]) > 0       # later steps: gates open somewhere
 
 
+@pytest.mark.parametrize("tie_rows,T", [(3000, 3000), (2600, 4000), (700, 4000)])
+def test_quantile_target_with_long_runs_of_equal_margins(tie_rows, T):
+    # tokens with all-zero hidden states have the same score 0.5 for every expert and the same cutoff, so their
+    # margins are exactly equal: more equal margins than the gathered lists hold (1024) send those experts down
+    # the path that walks the key scratch itself; fewer stay on the gather path.  Target bit-exact either way.
+    wl = synth.WORKLOADS["top3_single"].with_(T=T, H=128)
+    dev = "cuda"
+    x = synth.hidden_states(wl, 0, 0, dev)[None].contiguous()
+    x[0, :tie_rows] = 0
+    w = synth.router_weights(wl, 0, dev)[None].contiguous()
+    r = binding.Router(1, wl.E, wl.K, wl.H, wl.T, controller="quantile")
+    logits = torch.empty(1, T, wl.E, device=dev)
+    alpha = torch.empty(1, T, device=dev)
+    r.route_step(x, w, logits_out=logits, alpha_out=alpha)
+    r.controller_update()
+    r.poll()
+    bias = np_(r.load_stats()[1])[0]
+    want = oracle.quantile_target(np_(logits)[0], np_(alpha)[0], wl.K)
+    np.testing.assert_array_equal(bits(bias), bits(want))
+
+
 def test_quantile_target_count_property_on_gpu_result():
     # Section 2.3: with the cutoffs held fixed the new bias puts floor(mK/E)
     # (or, with ties at the cutoff, at most that many) margins strictly above zero
