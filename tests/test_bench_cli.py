@@ -5,6 +5,8 @@ import os
 import subprocess
 import sys
 
+import pytest
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -41,3 +43,21 @@ def test_reference_arm_prints_one_line_with_the_same_config_keys():
     r1 = _run(["--impl", "reference", "--workload", "tiny_top3", "--steps", "1", "--warmup", "0", "--gpus", "2"],
               env={"WORLD_SIZE": "2", "RANK": "1", "LOCAL_RANK": "1"})
     assert r1.returncode == 0 and r1.stdout.strip() == ""
+
+
+@pytest.mark.gpu
+def test_bench_line_has_the_contract_keys_on_a_small_workload():
+    r = _run(["--workload", "tiny_top3", "--steps", "5", "--warmup", "3", "--no-all-configs", "--min-region-s", "0.05",
+              "--ref-tokens-per-thread", "32"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks",
+                "near_tie", "all_configs", "repeats"):
+        assert key in line, key
+    assert line["n_gpus"] == 1 and line["steps"] == 5 and line["value"] > 0 and line["gpu_launches"] >= 10
+    assert line["config"]["workload"] == "tiny_top3" and line["vs_baseline"] is None
+    assert set(line["roofline"]) >= {"bound", "achieved", "peak", "unit", "frac", "traffic"}
+    assert line["e2e"]["h2d_bytes_per_step"] > 0 and line["e2e"]["d2h_bytes_per_step"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["near_tie"]["differing_with_clear_gap"] == 0

@@ -744,3 +744,45 @@ def test_full_size_deep_stack_layers():
 
 def test_full_size_large_scale_layers():
     _full_size(synth.WORKLOADS["top10_large"], layers=2, sample=256)
+
+
+@pytest.mark.parametrize("name", ["top10_deep", "top10_large"])
+def test_bench_launch_configuration_at_full_size(name):
+    # the whole configuration -- every layer at its full token count -- in ONE routing call without the dump, as
+    # the benchmark launches it (top10_large: 60 layers x 65536 tokens x hidden 4096 under chunk-split scheduling,
+    # 32 GB of hidden states): every token contributes exactly K counts, per-layer loads are the recount of the
+    # indices, indices are valid and distinct per token, gates sum to one, and a seeded row sample of every layer
+    # agrees with the fp64 definition (sets wherever the rank-K gap is clear, gates within 1e-5)
+    wl = synth.WORKLOADS[name]
+    dev = "cuda"
+    g = torch.Generator().manual_seed(wl.wid)
+    bias = (torch.randn(wl.L, wl.E, generator=g) * 0.01).contiguous()
+    x = torch.empty(wl.L, wl.T, wl.H, dtype=torch.bfloat16, device=dev)
+    for l in range(wl.L):
+        x[l] = synth.hidden_states(wl, l, 2, dev)
+    w = torch.stack([synth.router_weights(wl, l, dev) for l in range(wl.L)])
+    r = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T)
+    r.state_import(bias=bias.cuda())
+    idx, gate = r.route_step(x, w)
+    r.poll()
+    loads = np_(r.loads_peek())
+    assert loads.sum() == wl.L * wl.T * wl.K
+    ix, gt = np_(idx), np_(gate)
+    assert ix.min() >= 0 and ix.max() < wl.E
+    rng = np.random.default_rng(wl.wid)
+    differing = checked = 0
+    for l in range(wl.L):
+        np.testing.assert_array_equal(loads[l], np.bincount(ix[l].ravel(), minlength=wl.E))
+        srt = np.sort(ix[l], axis=1)
+        assert np.all(srt[:, 1:] != srt[:, :-1])                       # K distinct experts per token
+        np.testing.assert_allclose(gt[l].sum(axis=1), 1.0, atol=2e-6)
+        rows = np.sort(rng.choice(wl.T, 48, replace=False))
+        ref = oracle.route_tokens_f64(synth.bf16_bits(x[l][torch.from_numpy(rows).cuda()]), synth.bf16_bits(w[l]),
+                                      np_(bias[l]), wl.K, threads=THREADS)
+        same_set = np.all(np.sort(ix[l][rows], 1) == np.sort(ref["idx"], 1), axis=1)
+        assert np.all(same_set[ref["gap"] >= 1e-4])
+        same_order = np.all(ix[l][rows] == ref["idx"], axis=1)
+        assert np.max(np.abs(gt[l][rows][same_order] - ref["gate"][same_order])) <= 1e-5
+        differing += int((~same_set).sum())
+        checked += len(rows)
+    assert differing <= max(1, NEAR_TIE_BUDGET * checked)
