@@ -373,6 +373,30 @@ def test_quantile_controller_with_margin_histogram_estimate(bins, value_range, T
             assert np.max(np.abs(bias[l][inside].astype(np.float64) - exact[inside])) < h * (1 + 1e-6)
 
 
+def test_margin_histogram_estimate_with_exponential_moving_average():
+    # the EMA diagnostic of Section 3 on top of the histogram estimate: b = rho b + (1 - rho) Q_hist, three updates
+    # in a closed loop, bit for bit against the oracle's estimate and update
+    wl = synth.WORKLOADS["top3_single"].with_(T=1500, H=128, K=5)
+    dev, bins, value_range, rho = "cuda", 256, 1.0, 0.5
+    r = binding.Router(1, wl.E, wl.K, wl.H, wl.T, controller="quantile", qb_hist_bins=bins, qb_hist_range=value_range,
+                       qb_ema_rho=rho)
+    w = synth.router_weights(wl, 0, dev)[None].contiguous()
+    logits = torch.empty(1, wl.T, wl.E, device=dev)
+    alpha = torch.empty(1, wl.T, device=dev)
+    b = np.zeros(wl.E, np.float32)
+    ep = np.zeros(wl.E, np.float32)
+    for step in range(3):
+        x = synth.hidden_states(wl, 0, step, dev)[None].contiguous()
+        idx, gate = r.route_step(x, w, logits_out=logits, alpha_out=alpha)
+        r.controller_update()
+        r.poll()
+        loads, bias, _, _ = [np_(v) for v in r.load_stats()]
+        check_exact(np_(logits)[0], b, wl.K, np_(idx)[0], np_(gate)[0], np_(alpha)[0])
+        Q = oracle.quantile_target_hist(np_(logits)[0], np_(alpha)[0], wl.K, bins, value_range)
+        b, ep = oracle.quantile_update(b, ep, oracle.load_error(loads[0].astype(np.int64)), Q, rho=rho)
+        np.testing.assert_array_equal(bits(bias[0]), bits(b))
+
+
 def test_closed_loop_drifting_deep_stack_opens_the_derivative_gate():
     # deep-stack configuration at a reduced token count: the cluster means drift linearly over the 500 steps of
     # the workload, so consecutive controller steps taken from steps spread over the drift see the imbalance of
