@@ -199,7 +199,8 @@ int moe_gate_entropy(moe_route_ctx* ctx, const float* topk_gate, int32_t num_tok
  * in a fixed order in binary64: results are deterministic and agree with the
  * binary64 definition to about 1e-5 relative.
  * Forward statistics only: the gradient side of the auxiliary loss is a training-loop
- * matter.  Errors: MOE_ERR_INVALID_ARG (null logits, num_tokens < 1, aux without loads). */
+ * matter.  Errors: MOE_ERR_INVALID_ARG (null logits, logits not
+ * 16-byte aligned, num_tokens < 1, aux without loads). */
 int moe_score_stats(moe_route_ctx* ctx, const float* logits, int32_t num_tokens, const int32_t* loads,
                     float* entropy_biased, float* entropy_softmax, float* mean_prob, float* aux, void* cuda_stream);
 
@@ -241,6 +242,13 @@ int moe_route_poll(moe_route_ctx* ctx);
  * exact score of Section 2.2.  The filter is sound while this stays below half
  * of the slack compiled into the kernel (1e-5). */
 int moe_debug_score_gap(float* dev_result, void* cuda_stream);
+
+/* The same sweep for the quick score (hardware exponential and reciprocal
+ * approximations) with which the margin-histogram pass of the quantile
+ * controller bins a logit before deciding whether the exact score is needed:
+ * dev_result[0] = largest |quick - exact| over every finite fp32 logit.  The
+ * pass is exact while this stays below the gap compiled into it (3e-7). */
+int moe_debug_quick_score_gap(float* dev_result, void* cuda_stream);
 
 /* Quantile target without any allocation and without a context (the paper has
  * no counterpart for this call; it computes the same Q_j as the quantile

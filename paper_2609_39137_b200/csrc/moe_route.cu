@@ -29,6 +29,7 @@ struct Layout {
   size_t status, bias, e_prev, bias_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
   size_t qb_target, qb_hist, qb_prefix, qb_rank, qb_keys, qb_match, qb_fill, qb_list;
   size_t state_end;  // everything before this is cleared at init
+  size_t stat_cnt;   // [L] arrival counters of score_stats_finish_kernel (wrap to zero by themselves)
   size_t stat_P, stat_H, stat_aux, ent_part;   // per-CTA partial sums of moe_score_stats (written before they are read)
   size_t stage_x, stage_w, stage_idx, stage_gate;
   size_t w_t;   // [L][E][H] bf16 copy of the weights when they are given as [L][H][E]
@@ -80,6 +81,7 @@ Layout make_layout(const moe_route_config& c) {
   l.minvio = take((size_t)c.num_layers * 4);
   l.gate_count = take((size_t)c.num_layers * 4);
   l.qb_target = take(LE * 4);
+  l.stat_cnt = take((size_t)c.num_layers * 4);
   if (c.controller == MOE_CTRL_QUANTILE) {
     // exact selection: radix histogram [E][256]; histogram estimate: margin histogram [E][qb_hist_bins]
     l.qb_hist = take((size_t)c.num_experts * (c.qb_hist_bins > 0 ? c.qb_hist_bins : 256) * 4);
@@ -166,6 +168,7 @@ struct moe_route_ctx {
   int stall_next;       // moe_debug_route_stall: applies to the next routing launch only
   size_t merge_occ_smem;   // resident CTAs per SM of route_merge_kernel, cached per shared-memory size
   int merge_occ;
+  int qh_occ;              // resident CTAs per SM of qb_margin_hist_kernel (0: not asked yet)
   // cached TMA descriptors
   const void* map_x_ptr;
   const void* map_w_ptr;
@@ -509,12 +512,17 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
         attr_set[ctx->device & 63] = true;
       }
       const int groups = (c.num_experts + kQhCols - 1) / kQhCols;
-      const int per_sm = smem <= 33000 ? 6 : smem <= 66000 ? 3 : 1;
-      int splits = (per_sm * ctx->num_sms + groups - 1) / groups;
+      // one resident wave: every row split flushes its own copy of the non-empty bins, and a grid a little
+      // above what is resident runs a second, almost empty wave
+      if (ctx->qh_occ < 1) {
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, qb_margin_hist_kernel, kQhThreads, smem) != cudaSuccess || occ < 1)
+          occ = 1;
+        ctx->qh_occ = occ;
+      }
+      int splits = ctx->qh_occ * ctx->num_sms / groups;
       const int max_splits = (ctx->qb_tokens + 127) / 128;
       if (splits > max_splits) splits = max_splits;
-      const int min_splits = (ctx->qb_tokens + kQhMaxRowsPerCta - 1) / kQhMaxRowsPerCta;   // 16-bit counters per CTA
-      if (splits < min_splits) splits = min_splits;
       if (splits < 1) splits = 1;
       for (int l = 0; l < c.num_layers; ++l) {
         QhParams q{};
@@ -523,6 +531,7 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
         q.m = ctx->qb_tokens; q.E = c.num_experts; q.K = c.top_k; q.B = c.qb_hist_bins;
         q.range = c.qb_hist_range;
         q.inv_h = (float)c.qb_hist_bins / (2.0f * c.qb_hist_range);
+        q.edge_eps = qh_edge_eps(q.inv_h);
         q.hist = at<uint32_t>(ctx, ctx->lay.qb_hist);
         q.target = at<float>(ctx, ctx->lay.qb_target) + (size_t)l * c.num_experts;
         launch_chained(qb_margin_hist_kernel, dim3(groups, splits), dim3(kQhThreads), smem, st, q);
@@ -674,6 +683,7 @@ int moe_score_stats(moe_route_ctx* ctx, const float* logits, int32_t num_tokens,
   ctx->err[0] = 0;
   if (num_tokens < 1) return fail(ctx, MOE_ERR_INVALID_ARG, "num_tokens must be positive");
   if (aux && !loads) return fail(ctx, MOE_ERR_INVALID_ARG, "aux needs the loads of the same tokens");
+  if (reinterpret_cast<uintptr_t>(logits) % 16 != 0) return fail(ctx, MOE_ERR_INVALID_ARG, "logits must be 16-byte aligned");
   const moe_route_config& c = ctx->cfg;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   ctx->last_stream = st;
@@ -684,21 +694,33 @@ int moe_score_stats(moe_route_ctx* ctx, const float* logits, int32_t num_tokens,
   p.part_P = at<float>(ctx, ctx->lay.stat_P);
   p.part_H = at<float>(ctx, ctx->lay.stat_H);
   p.aux_part = at<double>(ctx, ctx->lay.stat_aux);
+  p.arrivals = at<unsigned int>(ctx, ctx->lay.stat_cnt);
   p.loads = loads; p.h_biased = entropy_biased; p.h_softmax = entropy_softmax; p.mean_prob = mean_prob; p.aux = aux;
   const dim3 grid(p.C, p.L);
-  if (p.E <= 256) launch_chained(score_stats_kernel<8>, grid, dim3(kStatThreads), 0, st, p);
-  else if (p.E <= 768) launch_chained(score_stats_kernel<24>, grid, dim3(kStatThreads), 0, st, p);
-  else launch_chained(score_stats_kernel<32>, grid, dim3(kStatThreads), 0, st, p);
+  {
+    const int nv = p.E <= 256 ? 2 : p.E <= 512 ? 4 : p.E <= 768 ? 6 : 8;
+    const bool full = (p.E == 128 * nv);
+    void (*kern)(StatParams) =
+        nv == 2 ? (full ? score_stats_kernel<2, true> : score_stats_kernel<2, false>)
+      : nv == 4 ? (full ? score_stats_kernel<4, true> : score_stats_kernel<4, false>)
+      : nv == 6 ? (full ? score_stats_kernel<6, true> : score_stats_kernel<6, false>)
+                : (full ? score_stats_kernel<8, true> : score_stats_kernel<8, false>);
+    static bool attr_set[64][8] = {};
+    bool& done = attr_set[ctx->device & 63][(nv / 2 - 1) * 2 + (full ? 1 : 0)];
+    if (!done) {
+      cudaError_t ae = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stat_smem_bytes(nv));
+      if (ae != cudaSuccess) return cuda_fail(ctx, ae, "cudaFuncSetAttribute(score_stats_kernel)");
+      done = true;
+    }
+    launch_chained(kern, grid, dim3(kStatThreads), stat_smem_bytes(nv), st, p);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_kernel launch");
   const int groups = (p.E + kStatFinExperts - 1) / kStatFinExperts;
   launch_chained(score_stats_finish_kernel, dim3(groups, p.L), dim3(1024), 0, st, p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_finish_kernel launch");
-  launch_chained(score_stats_scalar_kernel, dim3(p.L), dim3(32), 0, st, p, groups);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "score_stats_scalar_kernel launch");
-  ctx->launches += 3;
+  ctx->launches += 2;
   return MOE_OK;
 }
 
@@ -805,6 +827,32 @@ __global__ void score_gap_kernel(unsigned int* out) {
   }
   for (int d = 16; d > 0; d >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, d));
   if ((threadIdx.x & 31) == 0) atomicMax(out, __float_as_uint(worst));
+}
+
+__global__ void quick_score_gap_kernel(unsigned int* out) {
+  float worst = 0.0f;
+  const unsigned long long n = 1ull << 32;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned int bits = (unsigned int)i;
+    if ((bits & 0x7f800000u) == 0x7f800000u) continue;
+    const float z = __uint_as_float(bits);
+    worst = fmaxf(worst, fabsf(moe::quick_score(z) - moe::sigmoid_score(z)));
+  }
+  for (int d = 16; d > 0; d >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, d));
+  if ((threadIdx.x & 31) == 0) atomicMax(out, __float_as_uint(worst));
+}
+
+int moe_debug_quick_score_gap(float* dev_result, void* cuda_stream) {
+  if (!dev_result) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(dev_result, 0, sizeof(float), st) != cudaSuccess) return MOE_ERR_CUDA;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return MOE_ERR_CUDA;
+  quick_score_gap_kernel<<<sms * 8, 256, 0, st>>>(reinterpret_cast<unsigned int*>(dev_result));
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 int moe_debug_score_gap(float* dev_result, void* cuda_stream) {

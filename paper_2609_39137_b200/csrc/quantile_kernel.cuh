@@ -293,26 +293,26 @@ __global__ void __launch_bounds__(kQbSelectWarps * 32) qb_select_kernel(QbParams
 // the rule inside a bin are this library's choice).  One pass over the dump:
 //   bin k = floor((d + range) * inv_h) clamped to [0, B-1], d = sigmoid(z) - alpha
 //   (two rounded binary32 operations), B uniform bins over [-range, range);
-// the counts of a CTA's 16 experts are kept in shared memory as 16-bit halves of
-// 32-bit words ([B/2][expert] words, so the 16 lanes of a row hit 16 banks; a CTA sees fewer than 65536 rows, so a
-// half cannot carry into its neighbour; half the footprint of 32-bit counters,
-// twice the resident CTAs) and flushed with one global atomic per non-empty bin,
-// consecutive lanes on consecutive bins of one expert (contiguous addresses).  A second kernel (one warp
+// the counts of a CTA's 8 experts are kept in shared memory ([expert][B + 4] words, the 4 extra words skew the
+// experts' rows by four banks) and flushed with one global atomic per non-empty bin,
+// consecutive lanes on consecutive bins of one expert (contiguous addresses); the number of row splits is kept
+// small, because every split flushes its own copy of the non-empty bins.  A second kernel (one warp
 // per expert) finds the bin k* of the r-th smallest margin, r = m - floor(mK/E),
 // and interpolates in binary64: est = -range + (k* + ((r - below) - 0.5) / cnt) * h.
 // The counts are integers, so histograms of several ranks can be added before
 // the second kernel runs (that is what makes the estimate usable when the
 // tokens of a step are spread over data-parallel ranks).
-constexpr int kQhCols = 16;        // experts per CTA
-constexpr int kQhThreads = 256;
+constexpr int kQhCols = 8;         // experts per CTA: 32 bytes of a row, one DRAM sector
+constexpr int kQhThreads = 512;
 constexpr int kQhRowsInFlight = 8;
-constexpr int kQhMaxBins = 2048;   // 16 experts x 1024 words = 64 KB of shared memory
+constexpr int kQhMaxBins = 2048;   // 8 experts x 2052 words = 64 KB of shared memory
 
 struct QhParams {
   const float* logits;  // [m][E]
   const float* alpha;   // [m]
   int m, E, K, B;
   float range, inv_h;   // inv_h = (float)B / (2 * range)
+  float edge_eps;       // distance to a bin edge (in bins) below which the quick score is not trusted
   uint32_t* hist;       // [E][B], zero on entry of the histogram kernel, cleared again by the finish kernel
   float* target;        // [E] out: Q_j
 };
@@ -324,49 +324,91 @@ __device__ __forceinline__ int margin_bin(float d, float range, float inv_h, int
   return (fl >= (float)B) ? B - 1 : (int)fl;
 }
 
-__host__ __device__ inline size_t qh_smem_bytes(int B) { return (size_t)kQhCols * (B / 2) * 4; }
-constexpr int kQhMaxRowsPerCta = 65535;   // 16-bit counters
+// Quick score for binning: sigmoid(z) = 1 / (1 + 2^(-z log2 e)) with the hardware exponential and reciprocal
+// approximations.  Its distance to sigmoid_score is measured over every finite binary32 logit
+// (moe_debug_quick_score_gap) and stays below kQuickScoreGap; a margin whose quick bin position is closer than
+// that (scaled to bins, plus the rounding of the position itself) to an edge is binned again from the exact score.
+constexpr float kQuickScoreGap = 3e-7f;
+__device__ __forceinline__ float quick_score(float z) {
+  float u, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(u) : "f"(z * -1.44269504f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + u));
+  return r;
+}
+// In bins: the quick score's distance to the exact one, doubled, plus 3e-4 for the roundings that separate the two
+// positions (one of d + range, one of the product, one of the fused form, one of range * inv_h: each at most
+// half an ulp of a value below 2048, 6.1e-5).
+__host__ __device__ inline float qh_edge_eps(float inv_h) { return 2.0f * kQuickScoreGap * inv_h + 3e-4f; }
 
-// grid = (ceil(E / 16), row_splits); dynamic shared memory qh_smem_bytes(B).  A warp covers two rows of 16
-// experts (64 bytes each) per load; kQhRowsInFlight loads are issued before the first is used.
+__device__ __noinline__ int exact_margin_bin(float z, float a, float range, float inv_h, int B) {
+  return margin_bin(__fsub_rn(sigmoid_score(z), a), range, inv_h, B);
+}
+
+__host__ __device__ inline int qh_row_words(int B) { return B + 4; }
+__host__ __device__ inline size_t qh_smem_bytes(int B) { return (size_t)kQhCols * qh_row_words(B) * 4; }
+
+// grid = (ceil(E / 8), row_splits); dynamic shared memory qh_smem_bytes(B).  A lane takes four experts of a row
+// (one 16-byte load), a warp 16 rows of the CTA's 8 experts per load; kQhRowsInFlight loads are issued before the
+// first is used.  Every logit is binned from the quick score (two special-function instructions and about twenty
+// others); the few whose position is within edge_eps of a bin edge, and non-finite ones, are binned again with the
+// exact score chain, so the counts are those of the exact rule.
 __global__ void __launch_bounds__(kQhThreads) qb_margin_hist_kernel(QhParams p) {
   chained_launch_enter();
-  extern __shared__ uint32_t hs[];   // [B / 2][col] words, two 16-bit counters each
-  for (int i = threadIdx.x; i < kQhCols * (p.B / 2); i += kQhThreads) hs[i] = 0u;
+  extern __shared__ uint32_t hs[];   // [col][B + 4] counters
+  const int row_words = qh_row_words(p.B);
+  for (int i = threadIdx.x; i < kQhCols * row_words; i += kQhThreads) hs[i] = 0u;
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int c = lane & (kQhCols - 1), sub = lane >> 4;
-  const int col = blockIdx.x * kQhCols + c;
-  const bool live = col < p.E;
+  const int c0 = (lane & 1) * 4, sub = lane >> 1;         // first of the lane's four columns, row inside the warp's 16
+  const int col0 = blockIdx.x * kQhCols + c0;
+  const bool live = col0 < p.E;                           // E is a multiple of 4: a group is live or dead as a whole
   const int rows_per = (p.m + gridDim.y - 1) / gridDim.y;
   const int r0 = blockIdx.y * rows_per;
   const int r1 = min(p.m, r0 + rows_per);
-  constexpr int kRowsPerIter = (kQhThreads / 32) * 2;   // rows taken by the CTA per load
-  for (int i0 = r0 + warp * 2 + sub; i0 < r1; i0 += kRowsPerIter * kQhRowsInFlight) {
-    float z[kQhRowsInFlight], a[kQhRowsInFlight];
+  constexpr int kRowsPerIter = (kQhThreads / 32) * 16;    // rows taken by the CTA per load
+  constexpr float kMagic = 12582912.0f;                   // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
+  const float r_ih_half = p.range * p.inv_h - 0.5f;
+  const float trust = 0.5f - p.edge_eps;
+  uint32_t* my = hs + c0 * row_words;
+  for (int i0 = r0 + warp * 16 + sub; i0 < r1; i0 += kRowsPerIter * kQhRowsInFlight) {
+    float4 z[kQhRowsInFlight];
+    float a[kQhRowsInFlight];
 #pragma unroll
     for (int u = 0; u < kQhRowsInFlight; ++u) {
       const int i = i0 + u * kRowsPerIter;
       const bool ok = live && i < r1;
-      z[u] = ok ? __ldg(p.logits + (size_t)i * p.E + col) : 0.0f;
+      z[u] = ok ? __ldg(reinterpret_cast<const float4*>(p.logits + (size_t)i * p.E + col0)) : make_float4(0.f, 0.f, 0.f, 0.f);
       a[u] = ok ? __ldg(p.alpha + i) : 0.0f;
     }
 #pragma unroll
     for (int u = 0; u < kQhRowsInFlight; ++u) {
       const int i = i0 + u * kRowsPerIter;
       if (live && i < r1) {
-        const float d = __fsub_rn(sigmoid_score(z[u]), a[u]);
-        const int bin = margin_bin(d, p.range, p.inv_h, p.B);
-        atomicAdd(&hs[(bin >> 1) * kQhCols + c], 1u << (16 * (bin & 1)));
+        const float zz[4] = {z[u].x, z[u].y, z[u].z, z[u].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          // position in bins, minus 1/2, from the quick score; rounding it to the nearest integer is the floor
+          // of the position unless that lies close to an edge, which the test below catches (NaN included)
+          const float ph = fmaf(quick_score(zz[j]) - a[u], p.inv_h, r_ih_half);
+          const float tm = ph + kMagic;
+          const float off = ph - (tm - kMagic);                   // in [-1/2, 1/2]: distance to the bin's middle
+          int bin = __float_as_int(tm) - __float_as_int(kMagic);
+          bin = max(0, min(p.B - 1, bin));
+          if (!(fabsf(off) <= trust)) bin = exact_margin_bin(zz[j], a[u], p.range, p.inv_h, p.B);
+          atomicAdd(&my[j * row_words + bin], 1u);
+        }
       }
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < p.B * kQhCols; i += kQhThreads) {
-    const int cl = i / p.B, bin = i - cl * p.B;       // B is a multiple of 32: a warp stays inside one expert
+  // flush: a warp stays inside one expert, consecutive lanes on consecutive bins
+  for (int cl = 0; cl < kQhCols; ++cl) {
     const int cc = blockIdx.x * kQhCols + cl;
-    const uint32_t cnt = (hs[(bin >> 1) * kQhCols + cl] >> (16 * (bin & 1))) & 0xffffu;
-    if (cnt != 0u && cc < p.E) atomicAdd(&p.hist[(size_t)cc * p.B + bin], cnt);
+    if (cc >= p.E) break;
+    for (int bin = threadIdx.x; bin < p.B; bin += kQhThreads) {
+      const uint32_t cnt = hs[cl * row_words + bin];
+      if (cnt != 0u) atomicAdd(&p.hist[(size_t)cc * p.B + bin], cnt);
+    }
   }
 }
 

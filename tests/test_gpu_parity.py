@@ -166,6 +166,14 @@ def test_candidate_filter_slack_covers_every_fp32_logit():
     assert 0.0 < gap < 1e-5, gap
 
 
+def test_quick_score_gap_covers_every_fp32_logit():
+    # the margin-histogram pass bins a logit from a quick score (hardware exp2 and reciprocal approximations) and
+    # re-bins with the exact chain when the position is within twice the compiled gap (3e-7, scaled to bins) of an
+    # edge: over ALL finite fp32 logits the quick score must stay inside that gap
+    gap = binding.debug_quick_score_gap()
+    assert 0.0 < gap < 3e-7, gap
+
+
 # --------------------------------------------------------------- controllers
 def _drive(kind, L, E, K, steps, loads_fn, **cfg):
     r = binding.Router(L, E, K, 64, 128, controller=kind, ki=cfg.get("ki"), kd=cfg.get("kd"), eta=cfg.get("eta"),
@@ -553,6 +561,30 @@ def test_score_stats_match_oracle(L, T, H, E, K):
     only = r.score_stats(torch.from_numpy(res["logits"]).cuda())
     assert "aux" not in only
     np.testing.assert_array_equal(bits(np_(only["mean_prob"])), bits(np_(st["mean_prob"])))
+
+
+def test_score_stats_wide_logit_range():
+    # rows whose largest logit lies beyond +-40 take the kernel's direct sigmoid form, the others the shared-
+    # exponential form; both against the binary64 definition on a synthetic dump with row offsets up to +-70
+    L, T, E, K = 2, 900, 768, 10
+    rng = np.random.default_rng(23)
+    z = (rng.standard_normal((L, T, E)) * 3.0 + rng.uniform(-70.0, 70.0, size=(L, T, 1))).astype(np.float32)
+    assert (np.abs(z.max(axis=2)) > 40).mean() > 0.2 and (np.abs(z.max(axis=2)) <= 40).mean() > 0.2
+    bias = (rng.standard_normal((L, E)) * 0.2).astype(np.float32)
+    r = binding.Router(L, E, K, 64, T)
+    r.state_import(torch.from_numpy(bias).cuda(), torch.zeros(L, E, device="cuda"))
+    st = r.score_stats(torch.from_numpy(z).cuda())
+    r.poll()
+    for l in range(L):
+        hb = oracle.full_pool_entropy_mean(z[l], bias[l], "biased_sigmoid")
+        hs = oracle.full_pool_entropy_mean(z[l], None, "softmax")
+        _, P, _ = oracle.aux_loss_stats(z[l], np.zeros(E, dtype=np.int64))
+        assert abs(float(st["entropy_biased"][l]) - hb) <= 1e-5 * hb
+        assert abs(float(st["entropy_softmax"][l]) - hs) <= 1e-5 * hs
+        np.testing.assert_allclose(np_(st["mean_prob"][l]), P, rtol=1e-5, atol=1e-9)
+    raw = torch.zeros(L * T * E + 4, dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.MoeRouteError):                   # rows are read as 16-byte words
+        r.score_stats(raw[1:1 + L * T * E].view(L, T, E))
 
 
 def _fuzz_case(seed):
