@@ -412,6 +412,40 @@ def roofline_of(wl, total_ms, steps_total, route_ms, pk):
             "traffic": traffic, "traffic_note": traffic_note}
 
 
+def library_gemm_leg(wl, job, local_rank, seconds=1.5):
+    """Yardstick, not part of the path: the logits GEMM alone ([T x H] x [H x E] bf16 -> fp32-accumulated bf16
+    logits written to HBM, no score, no selection, no histogram) through torch.matmul on the job's own inputs,
+    layer after layer over the input ring, back to back for `seconds` under the same power cap, with the clock it
+    ran at.  What a fused routing step is worth is read against this on the same GPU: the library call still
+    needs a pass over its logits before it has routed anything."""
+    out = torch.empty(wl.T, wl.E, dtype=torch.bfloat16, device=job.dev)
+    wt = [job.w[l].t() for l in range(wl.L)]
+
+    def sweep(i):
+        x = job.xs[i % job.ring]
+        for l in range(wl.L):
+            torch.matmul(x[l], wt[l], out=out)
+    sweep(0)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n, t0 = 0, time.perf_counter()
+    e0.record()
+    while time.perf_counter() - t0 < seconds:
+        sweep(n)
+        n += 1
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / n
+    return {"what": "torch.matmul of the same [T x H] x [H x E] bf16 problem per layer on the same inputs, logits "
+                    "written as bf16, nothing routed; yardstick only",
+            "ms_per_step": ms, "tflops": 2.0 * wl.L * wl.T * wl.H * wl.E / ms / 1e9, "seconds": seconds,
+            "sm_mhz": clocks.get("sm_mhz"), "power_w": clocks.get("power_w")}
+
+
 def e2e_leg(wl, job, dev, world, steps_hint):
     """Same step through moe_route_step_host: pinned host x and W_r in, indices, gates and MaxVio/MinVio out,
     all copies inside the timed region."""
@@ -501,6 +535,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-configs", action="store_true", help="time only the chosen workload")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-library-gemm", action="store_true", help="skip the torch.matmul yardstick of the same problem")
     ap.add_argument("--chunk-split", type=int, default=0, choices=[0, 1, 2],
                     help="scheduling of the expert chunks (moe_route_config.chunk_split); 0 = the library chooses")
     ap.add_argument("--aux", action="store_true", help="time the calls outside the step (one GPU) and exit")
@@ -558,6 +593,9 @@ def main():
     loads, bias, maxvio, minvio = job.router.load_stats()
     gate_open = int(job.router.gate_stats().sum())
     breakdown = job.breakdown(max(3, min(args.steps, 24)))
+    lib_gemm = None
+    if rank == 0 and world == 1 and not args.no_library_gemm:
+        lib_gemm = library_gemm_leg(wl, job, local_rank)
     e2e = None
     if not args.no_e2e:
         e2e = e2e_leg(wl, job, dev, world, args.steps)
@@ -627,6 +665,11 @@ def main():
                 "roofline": headline_roofline, "cpu_baseline": cpu, "near_tie": near,
                 "gpu_launches": int(launches), "clocks": clocks, "breakdown": breakdown,
                 "last_step": last_step, "all_configs": others}
+        if lib_gemm:
+            # > 1: a whole routing step (logits, scores, top-K, gates, loads, controller) takes less time than
+            # the library's logits GEMM alone
+            lib_gemm["library_gemm_ms_over_routing_step_ms"] = lib_gemm["ms_per_step"] / (total_ms / steps_total)
+            line["library_gemm"] = lib_gemm
         if e2e:
             ms, n, wle, h2d, d2h, note = e2e
             line["e2e"] = {"value": wle.L * wl.T * world * n / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
