@@ -243,6 +243,24 @@ int moe_route_poll(moe_route_ctx* ctx);
  * of the slack compiled into the kernel (1e-5). */
 int moe_debug_score_gap(float* dev_result, void* cuda_stream);
 
+/* Validation utility for the reciprocal inside the score chain (Section 2.2: the
+ * score ends in a correctly rounded reciprocal).  The kernels compute it as the
+ * hardware approximation plus one Newton step with an exact residual instead of
+ * the math library's routine.  Sweeps all 2^32 fp32 bit patterns and writes two
+ * counters to dev_result (device, two uint32): [0] logits whose score differs in
+ * any bit between the two reciprocals, [1] normal numbers d with |d| in
+ * [2^-126, 2^126] whose reciprocal differs.  Both must be 0. */
+int moe_debug_rcp_check(uint32_t* dev_result, void* cuda_stream);
+
+/* Validation utility for the gate division (Eq. 3: g = s / sum of the selected
+ * s, correctly rounded).  The kernels divide by multiplying with the correctly
+ * rounded reciprocal of the denominator and correcting twice with exact
+ * residuals.  Compares that with the math library's correctly rounded division
+ * for every fp32 denominator in [2^-20, 32] with 48 numerators each (about 1e10
+ * pairs) and writes the number of differing pairs to dev_result[0] (device, one
+ * uint32).  Must be 0. */
+int moe_debug_division_check(uint32_t* dev_result, void* cuda_stream);
+
 /* The same sweep for the quick score (hardware exponential and reciprocal
  * approximations) with which the margin-histogram pass of the quantile
  * controller bins a logit before deciding whether the exact score is needed:

@@ -25,7 +25,7 @@ CONTROLLERS = {"id": MOE_CTRL_ID, "fixed_step": MOE_CTRL_FIXED_STEP, "quantile":
 SYMBOLS = ["moe_route_default_config", "moe_route_workspace_bytes", "moe_route_init", "moe_route_step",
            "moe_route_step_host", "moe_controller_update", "moe_load_stats", "moe_gate_stats", "moe_loads_peek",
            "moe_loads_add", "moe_loads_buffer", "moe_state_export", "moe_state_import", "moe_route_poll", "moe_route_launch_count",
-           "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_debug_quick_score_gap", "moe_quantile_target_static",
+           "moe_last_error", "moe_route_destroy", "moe_debug_score_gap", "moe_debug_quick_score_gap", "moe_debug_rcp_check", "moe_debug_division_check", "moe_quantile_target_static",
            "moe_load_diagnostics", "moe_gate_entropy", "moe_debug_wait_timeout", "moe_score_stats", "moe_debug_route_stall", "moe_debug_build"]
 
 
@@ -82,6 +82,8 @@ def load():
     L.moe_route_destroy.argtypes = [vp]
     L.moe_debug_score_gap.argtypes = [vp, vp]
     L.moe_debug_quick_score_gap.argtypes = [vp, vp]
+    L.moe_debug_rcp_check.argtypes = [vp, vp]
+    L.moe_debug_division_check.argtypes = [vp, vp]
     L.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
     L.moe_debug_route_stall.argtypes = [vp, i32]
     L.moe_debug_build.argtypes = []
@@ -112,6 +114,27 @@ def debug_score_gap(device="cuda") -> float:
     if rc != MOE_OK:
         raise MoeRouteError(rc, "moe_debug_score_gap failed")
     return float(out.item())
+
+
+def debug_rcp_check(device="cuda"):
+    """(scores, reciprocals) that differ between the kernels' branch-free reciprocal and the library's correctly
+    rounded one, over all 2^32 fp32 bit patterns (runs on the GPU); both must be 0."""
+    out = torch.zeros(2, dtype=torch.int32, device=device)
+    rc = load().moe_debug_rcp_check(_ptr(out), _stream())
+    if rc != MOE_OK:
+        raise MoeRouteError(rc, "moe_debug_rcp_check failed")
+    a, b = out.tolist()
+    return a, b
+
+
+def debug_division_check(device="cuda") -> int:
+    """Pairs (numerator, denominator) for which the kernels' gate division differs from the library's correctly
+    rounded division, over every fp32 denominator in [2^-20, 32] with 48 numerators each; must be 0."""
+    out = torch.zeros(1, dtype=torch.int32, device=device)
+    rc = load().moe_debug_division_check(_ptr(out), _stream())
+    if rc != MOE_OK:
+        raise MoeRouteError(rc, "moe_debug_division_check failed")
+    return int(out.item())
 
 
 def debug_quick_score_gap(device="cuda") -> float:

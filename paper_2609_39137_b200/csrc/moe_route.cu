@@ -829,6 +829,81 @@ __global__ void score_gap_kernel(unsigned int* out) {
   if ((threadIdx.x & 31) == 0) atomicMax(out, __float_as_uint(worst));
 }
 
+// out[0]: number of binary32 inputs (all 2^32 bit patterns) for which the score chain with the branch-free
+// reciprocal differs in any bit from the chain with the library's correctly rounded reciprocal;
+// out[1]: number of normal d in [2^-126, 2^126] for which rcp_rn_normal(d) differs from __frcp_rn(d)
+__global__ void rcp_check_kernel(unsigned int* out) {
+  unsigned int bad_score = 0, bad_rcp = 0;
+  const unsigned long long n = 1ull << 32;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned int bits = (unsigned int)i;
+    const float z = __uint_as_float(bits);
+    if (__float_as_uint(moe::sigmoid_score_t<false>(z)) != __float_as_uint(moe::sigmoid_score_t<true>(z))) bad_score += 1;
+    const unsigned int ex = (bits >> 23) & 0xffu;
+    if (ex >= 1u && ex <= 252u && !(ex == 252u && (bits & 0x7fffffu) != 0u)) {     // |d| in [2^-126, 2^126]
+      if (__float_as_uint(moe::rcp_rn_normal(z)) != __float_as_uint(__frcp_rn(z))) bad_rcp += 1;
+    }
+  }
+  for (int d = 16; d > 0; d >>= 1) {
+    bad_score += __shfl_xor_sync(0xffffffffu, bad_score, d);
+    bad_rcp += __shfl_xor_sync(0xffffffffu, bad_rcp, d);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    if (bad_score) atomicAdd(&out[0], bad_score);
+    if (bad_rcp) atomicAdd(&out[1], bad_rcp);
+  }
+}
+
+int moe_debug_rcp_check(uint32_t* dev_result, void* cuda_stream) {
+  if (!dev_result) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(dev_result, 0, 2 * sizeof(uint32_t), st) != cudaSuccess) return MOE_ERR_CUDA;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return MOE_ERR_CUDA;
+  rcp_check_kernel<<<sms * 8, 256, 0, st>>>(dev_result);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+// out[0]: pairs (a, b) for which div_rn_by differs from __fdiv_rn.  b runs over every binary32 number in
+// [2^-20, 32]; for each b, 48 numerators a in (0, b]: b scaled by factors just below 1 and by pseudo-random
+// factors over 40 binades (the shapes a gate has: one score over a sum that contains it).
+__global__ void division_check_kernel(unsigned int* out) {
+  unsigned int bad = 0;
+  const unsigned int b_lo = 0x35800000u /* 2^-20 */, b_hi = 0x42000000u /* 32 */;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x + b_lo; i <= b_hi;
+       i += (unsigned long long)gridDim.x * blockDim.x) {
+    const float b = __uint_as_float((unsigned int)i);
+    const float r = moe::rcp_rn_normal(b);
+    unsigned int h = (unsigned int)i * 2654435761u + 12345u;
+    for (int k = 0; k < 48; ++k) {
+      h = h * 1664525u + 1013904223u;
+      float a;
+      if (k < 8) a = b * (1.0f - (float)k * 5.9604645e-8f);                       // just below b
+      else if (k < 16) a = __uint_as_float(((unsigned int)i & 0xff800000u) | (h >> 9));   // same binade, random mantissa
+      else a = b * __uint_as_float(((87u + (h >> 27)) << 23) | (h & 0x7fffffu));  // b * [2^-40, 2^-8)
+      if (!(a > 0.0f) || a > b || !moe::gate_division_safe(a, b)) continue;
+      if (__float_as_uint(moe::div_rn_by(a, b, r)) != __float_as_uint(__fdiv_rn(a, b))) bad += 1;
+    }
+  }
+  for (int d = 16; d > 0; d >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, d);
+  if ((threadIdx.x & 31) == 0 && bad) atomicAdd(&out[0], bad);
+}
+
+int moe_debug_division_check(uint32_t* dev_result, void* cuda_stream) {
+  if (!dev_result) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(dev_result, 0, sizeof(uint32_t), st) != cudaSuccess) return MOE_ERR_CUDA;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return MOE_ERR_CUDA;
+  division_check_kernel<<<sms * 8, 256, 0, st>>>(dev_result);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
 __global__ void quick_score_gap_kernel(unsigned int* out) {
   float worst = 0.0f;
   const unsigned long long n = 1ull << 32;

@@ -137,10 +137,20 @@ __global__ void __launch_bounds__(kMergeThreads, 3) route_merge_kernel(const Mer
     }
     // every entry of the row has been read: the row now takes the outputs, (expert, gate) at position k
     float2* out_row = warp_s + lane * stride;
+    // one reciprocal of the denominator and a branch-free correctly rounded division per gate; a token whose
+    // denominator or smallest score is outside the range where that holds takes the library's division
+    float smin = INFINITY;
+#pragma unroll
+    for (int k = 0; k < kMergeMaxK; ++k)
+      if (k < p.K) smin = fminf(smin, sel_s[k]);
+    const bool safe = gate_division_safe(smin, denom);
+    const float rden = rcp_rn_normal(safe ? denom : 1.0f);
 #pragma unroll
     for (int k = 0; k < kMergeMaxK; ++k) {
       if (k < p.K) {
-        out_row[k] = make_float2(__int_as_float(sel_e[k]), (denom == 0.0f) ? uniform : __fdiv_rn(sel_s[k], denom));
+        float gk = div_rn_by(sel_s[k], denom, rden);
+        if (!safe) gk = (denom == 0.0f) ? uniform : __fdiv_rn(sel_s[k], denom);
+        out_row[k] = make_float2(__int_as_float(sel_e[k]), gk);
         if ((unsigned)sel_e[k] < (unsigned)p.E) atomicAdd(&hist_s[sel_e[k]], 1);
       }
     }

@@ -166,6 +166,20 @@ def test_candidate_filter_slack_covers_every_fp32_logit():
     assert 0.0 < gap < 1e-5, gap
 
 
+def test_branch_free_reciprocal_equals_the_correctly_rounded_one_everywhere():
+    # the score chain ends in a correctly rounded reciprocal (Section 2.2 as read here); the kernels take the
+    # hardware approximation plus one Newton step: over ALL 2^32 logits the score has the same bits as with the
+    # math library's reciprocal, and so has the reciprocal of every normal number with a normal reciprocal
+    assert binding.debug_rcp_check() == (0, 0)
+
+
+def test_gate_division_equals_the_correctly_rounded_one():
+    # gates are s / D correctly rounded (Eq. 3 as read here); the kernels multiply by the correctly rounded 1 / D and
+    # correct twice with exact residuals: same bits as the library's division for every denominator in [2^-20, 32]
+    # with 48 numerators each
+    assert binding.debug_division_check() == 0
+
+
 def test_quick_score_gap_covers_every_fp32_logit():
     # the margin-histogram pass bins a logit from a quick score (hardware exp2 and reciprocal approximations) and
     # re-bins with the exact chain when the position is within twice the compiled gap (3e-7, scaled to bins) of an
