@@ -95,22 +95,24 @@ __global__ void __launch_bounds__(kMergeThreads, 3) route_merge_kernel(const Mer
     __syncwarp();
     const int tok = tok0 + lane;
     if (lane < rows) {
+    // Heads of the (up to four) lists; a step picks the best head by a two-round tournament and replaces it
+    // with its list's next entry.  Everything is selections under predicates: lanes differ in which list wins,
+    // and a branch per list would run all four bodies one after the other in every step.
     float hv[kMergeMaxChunks], hs[kMergeMaxChunks];
-    int he[kMergeMaxChunks], pos[kMergeMaxChunks];
-#pragma unroll
-    for (int c = 0; c < kMergeMaxChunks; ++c) pos[c] = 0;
-    auto load_head = [&](int c) {
+    int he[kMergeMaxChunks];
+    uint32_t pos_all = 0;                                    // four 8-bit positions
+    auto entry = [&](int c, int pos, float& v, float& sc, int& e) {
       // an exhausted list, an entry without an expert and a padding column all rank after every real entry
-      float2 se = make_float2(0.0f, __int_as_float(0x7fffffff));
-      if (c < p.num_chunks && pos[c] < p.cand_len) se = mine[c * p.cand_len + pos[c]];
-      const int e = __float_as_int(se.y);
-      const bool real = (unsigned)e < (unsigned)p.E;
-      hs[c] = se.x;
-      he[c] = real ? e : 0x7fffffff;
-      hv[c] = real ? __fadd_rn(se.x, bias_s[e]) : -INFINITY;
+      const bool in = c < p.num_chunks && pos < p.cand_len;
+      const float2 se = mine[min(c, p.num_chunks - 1) * p.cand_len + min(pos, p.cand_len - 1)];
+      const int ei = __float_as_int(se.y);
+      const bool real = in && (unsigned)ei < (unsigned)p.E;
+      sc = se.x;
+      e = real ? ei : 0x7fffffff;
+      v = real ? __fadd_rn(se.x, bias_s[real ? ei : 0]) : -INFINITY;
     };
 #pragma unroll
-    for (int c = 0; c < kMergeMaxChunks; ++c) load_head(c);
+    for (int c = 0; c < kMergeMaxChunks; ++c) entry(c, 0, hv[c], hs[c], he[c]);
     float alpha = __int_as_float(0x7fc00000);
     float denom = 0.0f;
     float sel_s[kMergeMaxK];
@@ -118,21 +120,28 @@ __global__ void __launch_bounds__(kMergeThreads, 3) route_merge_kernel(const Mer
 #pragma unroll
     for (int k = 0; k < kMergeMaxK + 1; ++k) {
       if (k < p.cand_len) {                                // rank K is only needed for alpha
-        int best = 0;
-        float bv = hv[0], bs = hs[0];
-        int be = he[0];
-#pragma unroll
-        for (int c = 1; c < kMergeMaxChunks; ++c)
-          if (ranks_before(hv[c], he[c], bv, be)) { best = c; bv = hv[c]; bs = hs[c]; be = he[c]; }
+        float v01, s01, v23, s23, bv, bs;
+        int e01, e23, be;
+        const bool t01 = ranks_before(hv[1], he[1], hv[0], he[0]);
+        const bool t23 = ranks_before(hv[3], he[3], hv[2], he[2]);
+        select_triple(t01, hv[0], hv[1], hs[0], hs[1], he[0], he[1], v01, s01, e01);
+        select_triple(t23, hv[2], hv[3], hs[2], hs[3], he[2], he[3], v23, s23, e23);
+        const bool tb = ranks_before(v23, e23, v01, e01);
+        select_triple(tb, v01, v23, s01, s23, e01, e23, bv, bs, be);
+        const int best = tb ? (t23 ? 3 : 2) : (t01 ? 1 : 0);
         if (k < kMergeMaxK && k < p.K) {
           sel_s[k] = bs;
           sel_e[k] = be;
           denom = (k == 0) ? bs : __fadd_rn(denom, bs);     // D = ((s_0 + s_1) + s_2) + ... in output order
         }
         if (k == p.K) alpha = bv;
+        const int npos = (int)((pos_all >> (8 * best)) & 0xffu) + 1;
+        pos_all += 1u << (8 * best);
+        float nv, ns;
+        int ne;
+        entry(best, npos, nv, ns, ne);
 #pragma unroll
-        for (int c = 0; c < kMergeMaxChunks; ++c)
-          if (best == c) { pos[c] += 1; load_head(c); }
+        for (int c = 0; c < kMergeMaxChunks; ++c) select_triple(best == c, hv[c], nv, hs[c], ns, he[c], ne, hv[c], hs[c], he[c]);
       }
     }
     // every entry of the row has been read: the row now takes the outputs, (expert, gate) at position k
