@@ -100,6 +100,26 @@ def test_route_operand_layout_one_hot():
     full_check(res, K)
 
 
+@pytest.mark.parametrize("chunk_split", [1, 2])
+def test_tiny_scores_take_the_library_division(chunk_split):
+    # logits of -72 .. -88: every score is below 2^-100, where the kernels' branch-free gate division is not
+    # used (library division instead), the approximate score is 0 for every column (all within the filter slack:
+    # the exact insertion lists do the work), and one-hot router rows over 256 hidden columns give every logit
+    # three times (exact ties, lowest index wins).  Gates are ratios of numbers near 1e-35.
+    T, H, E, K = 300, 256, 768, 10
+    dev = "cuda"
+    g = torch.Generator().manual_seed(77)
+    x = (-(72.0 + 16.0 * torch.rand(1, T, H, generator=g))).to(torch.bfloat16).to(dev)
+    w = torch.zeros(1, E, H, device=dev, dtype=torch.bfloat16)
+    hsel = (torch.arange(E, device=dev) * 7 + 3) % H
+    w[0, torch.arange(E, device=dev), hsel] = 1.0
+    res = route_once(T, H, E, K, x=x, w=w, want_alpha=True, chunk_split=chunk_split)
+    np.testing.assert_array_equal(res["logits"][0], np_(x[0].float()[:, hsel]))
+    assert res["logits"].max() < -69.4            # sigmoid < 2^-100
+    full_check(res, K)
+    assert np.all(np.abs(res["gate"].sum(axis=-1) - 1.0) < 1e-5)
+
+
 def test_route_exact_ties_pick_lowest_index():
     # all-zero hidden states: every logit is 0, every score 0.5 -> with zero
     # bias the K lowest indices win; with a bias plateau the plateau's lowest
