@@ -53,10 +53,10 @@ L2_BYTES = 126e6
 NCU_TRAFFIC = {
     # routing kernel read + write, merge kernel read + write (2 of the 60 layers: a capture of the full launch
     # would hold 64 GB on the device under the profiler)
-    "top10_large": {"bytes": 1135516000 + 77426944 + 31525120 + 768, "layers": 2,
+    "top10_large": {"bytes": 1148419000 + 79036672 + 31513088 + 256, "layers": 2,
                     "profile": "profiles/route_step_kernel_top10_large.md"},
-    "top10_single": {"bytes": 71075840 + 3006976, "layers": 1, "profile": "profiles/route_step_kernel_top10_single.md"},
-    "top10_deep": {"bytes": 329697792 + 17890816, "layers": 4, "profile": "profiles/route_step_kernel_top10_deep_4layers.md"},
+    "top10_single": {"bytes": 70553344 + 2378496, "layers": 1, "profile": "profiles/route_step_kernel_top10_single.md"},
+    "top10_deep": {"bytes": 332765952 + 18158848, "layers": 4, "profile": "profiles/route_step_kernel_top10_deep_4layers.md"},
 }
 
 
