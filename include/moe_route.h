@@ -95,7 +95,9 @@ typedef struct {
                            rows in its epilogue; 2 = the chunks of a tile go to different CTA pairs that run at
                            the same time (the tile is streamed from HBM once) and a merge kernel finishes the
                            rows from L*ceil(E/256)*max_tokens*(K+1)*8 bytes of workspace; 0 = chosen by the
-                           hidden size (2 when the tiles of all resident pairs no longer fit in L2) */
+                           library: 2 when the tiles of all resident pairs no longer fit in L2 (hidden > 3072)
+                           or when L*ceil(max_tokens/256)*ceil(E/256) <= 64, i.e. every (tile, chunk) gets a
+                           CTA pair of its own; else 1 */
   int32_t qb_hist_bins; /* MOE_CTRL_QUANTILE only.  0 = exact quantile of Eq. 7 (radix select over the dump).
                            B > 0 (multiple of 32, 32..2048) = the estimate the footnote to Eq. 7 mentions for use
                            at scale, from a per-expert margin histogram -- the paper fixes neither bins nor

@@ -48,12 +48,16 @@ constexpr unsigned char kCanaryByte = 0xC5;
 // Chunk-split scheduling (the expert chunks of a token tile go to different CTA pairs, a merge kernel
 // finishes): chosen when one CTA pair re-reading its tile once per chunk would push the tiles of all
 // resident pairs out of L2 -- 74 pairs x 256 tokens x hidden x 2 bytes exceeds the 126 MB L2 beyond
-// hidden ~ 3300 -- and there is more than one chunk.
+// hidden ~ 3300 -- and there is more than one chunk.  Also chosen for launches so small that every (tile, chunk)
+// gets a CTA pair of its own (at most 64 such items at max_tokens): the chunks of a tile are then scanned side by
+// side instead of one after the other, which is worth more than the merge launch costs.
 bool use_chunk_split(const moe_route_config& c) {
   if (c.num_experts <= kBN) return false;
   if (c.chunk_split == 1) return false;
   if (c.chunk_split == 2) return true;
-  return c.hidden > 3072;
+  const long long chunks = (c.num_experts + kBN - 1) / kBN;
+  const long long tile_pairs = ((long long)c.max_tokens + 2 * kBM - 1) / (2 * kBM);
+  return c.hidden > 3072 || (long long)c.num_layers * tile_pairs * chunks <= 64;
 }
 
 Layout make_layout(const moe_route_config& c) {
