@@ -44,6 +44,10 @@ METRIC = "routed_tokens_per_s"
 UNIT = "tokens/s"
 HEADLINE = "top10_large"
 OTHERS = ["tiny_top3", "top10_single", "top3_single", "top5_single", "top10_deep", "top8_of_256"]
+# the baseline controllers on the Top-3 workload (the third configuration compares three controllers): the fixed-step
+# integral costs what the ID update costs; Quantile Balancing needs the logits dump and the per-token threshold
+# from the routing kernel and a selection pass over the dump in the update
+CONTROLLER_VARIANTS = [("top3_single", "fixed_step"), ("top3_single", "quantile")]
 L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the routing kernels of one moe_route_step, per launch, from ncu
@@ -273,8 +277,9 @@ class Job:
 
     chunk_split = 0      # moe_route_config.chunk_split of every context made here (0 = the library chooses)
 
-    def __init__(self, wl, dev, rank, world, dist):
+    def __init__(self, wl, dev, rank, world, dist, controller="id"):
         from paper_2609_39137_b200 import binding, dp
+        self.controller = controller
         self.wl, self.dev, self.dist, self.dp = wl, dev, dist, dp
         self.ring = ring_size(wl)
         # seeded, synthetic; each rank draws its own token shard (step index offset by the rank)
@@ -287,11 +292,16 @@ class Job:
             self.xs.append(x)
         self.idx = torch.empty(wl.L, wl.T, wl.K, dtype=torch.int32, device=dev)
         self.gate = torch.empty(wl.L, wl.T, wl.K, dtype=torch.float32, device=dev)
-        self.router = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T, controller="id", device=dev,
+        self.router = binding.Router(wl.L, wl.E, wl.K, wl.H, wl.T, controller=controller, device=dev,
                                      chunk_split=Job.chunk_split)
+        self.logits = self.alpha = None
+        if controller == "quantile":     # Eq. 7 needs every token's scores and its threshold
+            self.logits = torch.empty(wl.L, wl.T, wl.E, dtype=torch.float32, device=dev)
+            self.alpha = torch.empty(wl.L, wl.T, dtype=torch.float32, device=dev)
 
     def step(self, i):
-        self.router.route_step(self.xs[i % self.ring], self.w, self.idx, self.gate)
+        self.router.route_step(self.xs[i % self.ring], self.w, self.idx, self.gate, logits_out=self.logits,
+                               alpha_out=self.alpha)
         if self.dist is not None:
             self.dp.allreduce_loads(self.router, self.dist)   # Algorithm 1 line 4: counts summed over the DP group
         self.router.controller_update()
@@ -339,7 +349,8 @@ class Job:
                 probe = ev.get(i)
                 if probe is not None:
                     probe[0].record()
-                self.router.route_step(self.xs[i % self.ring], self.w, self.idx, self.gate)
+                self.router.route_step(self.xs[i % self.ring], self.w, self.idx, self.gate, logits_out=self.logits,
+                                       alpha_out=self.alpha)
                 if probe is not None:
                     probe[1].record()
                 if self.dist is not None:
@@ -360,7 +371,8 @@ class Job:
         bev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_break)]
         for i in range(n_break):
             bev[i][0].record()
-            self.router.route_step(self.xs[i % self.ring], self.w, self.idx, self.gate)
+            self.router.route_step(self.xs[i % self.ring], self.w, self.idx, self.gate, logits_out=self.logits,
+                                   alpha_out=self.alpha)
             bev[i][1].record()
             if self.dist is not None:
                 self.dp.allreduce_loads(self.router, self.dist)
@@ -618,11 +630,13 @@ def main():
     # ---- the other configurations, briefly (same run, same rules; one entry each)
     others = []
     if not args.no_all_configs and args.layers == 0:
-        for name in OTHERS:
-            if name == wl.name:
+        for name, ctrl in [(n, "id") for n in OTHERS] + CONTROLLER_VARIANTS:
+            if name == wl.name and ctrl == "id":
                 continue
+            if ctrl == "quantile" and world > 1:
+                continue          # Eq. 7 ranks the tokens of one rank's dump; not a data-parallel configuration here
             o = synth.WORKLOADS[name]
-            oj = Job(o, dev, rank, world, dist)
+            oj = Job(o, dev, rank, world, dist, controller=ctrl)
             o_est = oj.prewarm(0.2, 3)
             o_steps = max(3, args.steps)
             o_rep = max(1, math.ceil(args.min_region_s * 1e3 / max(1e-6, o_est * o_steps)))
@@ -637,7 +651,7 @@ def main():
                 o_ms = float(t[0])
             if rank == 0:
                 rf = roofline_of(o, o_ms, o_steps * o_rep, o_route, pk)
-                others.append({"workload": name, "L": o.L, "T": o.T, "H": o.H, "E": o.E, "K": o.K,
+                others.append({"workload": name, "controller": ctrl, "L": o.L, "T": o.T, "H": o.H, "E": o.E, "K": o.K,
                                "steps": o_steps, "repeats": o_rep, "timed_region_s": o_ms * 1e-3,
                                "ms_per_step": o_ms / (o_steps * o_rep),
                                "tokens_per_s": o.L * o.T * world * o_steps * o_rep / (o_ms * 1e-3),

@@ -27,7 +27,7 @@ constexpr size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign;
 
 struct Layout {
   size_t status, bias, e_prev, bias_prev, loads_acc, loads_last, maxvio, minvio, gate_count;
-  size_t qb_target, qb_hist, qb_prefix, qb_rank, qb_keys, qb_match, qb_fill, qb_list;
+  size_t qb_target, qb_hist, qb_prefix, qb_rank, qb_keys, qb_match, qb_fill, qb_list, qb_deep;
   size_t state_end;  // everything before this is cleared at init
   size_t stat_cnt;   // [L] arrival counters of score_stats_finish_kernel (wrap to zero by themselves)
   size_t stat_P, stat_H, stat_aux, ent_part;   // per-CTA partial sums of moe_score_stats (written before they are read)
@@ -98,6 +98,7 @@ Layout make_layout(const moe_route_config& c) {
     l.qb_match = take((size_t)c.num_experts * 4);
     l.qb_fill = take((size_t)c.num_experts * 4);
     l.qb_list = take((size_t)c.num_experts * kQbListCap * 2);
+    l.qb_deep = take(4);
   }
   {
     const size_t LC = (size_t)c.num_layers * stat_ctas_per_layer(c.num_layers);
@@ -565,8 +566,11 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
       q.match = at<uint32_t>(ctx, ctx->lay.qb_match);
       q.fill = at<uint32_t>(ctx, ctx->lay.qb_fill);
       q.list = at<uint16_t>(ctx, ctx->lay.qb_list);
+      q.deep = at<uint32_t>(ctx, ctx->lay.qb_deep);
       launch_chained(qb_init_kernel, dim3(64), dim3(256), 0, st, q);
-      for (int pass = 0; pass < 2; ++pass) {
+      // two digit passes; the third one's kernels return at once unless the second scan found a set that does not
+      // fit the list
+      for (int pass = 0; pass < 3; ++pass) {
         launch_chained(qb_hist_kernel, dim3(col_groups, splits), dim3(kQbThreads), 0, st, q, pass);
         launch_chained(qb_scan_kernel, dim3((c.num_experts * 32 + 255) / 256), dim3(256), 0, st, q, pass);
       }
@@ -574,7 +578,7 @@ int moe_controller_update(moe_route_ctx* ctx, void* cuda_stream) {
       launch_chained(qb_gather_kernel, dim3(col_groups, splits), dim3(kQbThreads), 0, st, q);
       launch_chained(qb_select_kernel, dim3((c.num_experts + kQbSelectWarps - 1) / kQbSelectWarps),
                      dim3(kQbSelectWarps * 32), 0, st, q);
-      ctx->launches += 7;
+      ctx->launches += 9;
     }
     {
       cudaError_t qe = cudaGetLastError();

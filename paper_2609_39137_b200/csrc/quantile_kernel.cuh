@@ -49,6 +49,10 @@ struct QbParams {
   uint32_t* match;      // [E] number of keys sharing the prefix (the count of the bin chosen by the second scan)
   uint32_t* fill;       // [E] entries gathered so far
   uint16_t* list;       // [E][kQbListCap] low 16 bits of the gathered keys
+  // Margins with a large common offset (a bias that has drifted as a whole) share their sign, exponent and leading
+  // mantissa bits, so the keys that share a 16-bit prefix can be many more than a list holds; the second scan then
+  // raises this flag and a third digit pass runs before the gather (its two kernels return at once otherwise)
+  uint32_t* deep;       // [1] or null
 };
 constexpr int kQbListCap = 1024;
 
@@ -74,12 +78,14 @@ __global__ void qb_init_kernel(QbParams p) {
     p.prefix[j] = 0u;
     p.rank[j] = (uint32_t)r;
   }
+  if (j == 0 && p.deep != nullptr) *p.deep = 0u;
   for (int i = j; i < p.E * 256; i += gridDim.x * blockDim.x) p.hist[i] = 0u;
 }
 
 // pass = 0..3, most significant byte first.  grid = (ceil(E/32), row_splits)
 __global__ void __launch_bounds__(kQbThreads) qb_hist_kernel(QbParams p, int pass) {
   chained_launch_enter();
+  if (p.deep != nullptr && pass == 2 && *p.deep == 0u) return;   // the third digit is not needed
   __shared__ uint32_t h[256 * kQbCols];  // [bin][col]: lanes hit distinct banks
   for (int i = threadIdx.x; i < 256 * kQbCols; i += kQbThreads) h[i] = 0u;
   __syncthreads();
@@ -144,6 +150,7 @@ __global__ void __launch_bounds__(kQbThreads) qb_hist_kernel(QbParams p, int pas
 // digit, clear the histogram; after the last pass emit Q_j = -margin.
 __global__ void qb_scan_kernel(QbParams p, int pass) {
   chained_launch_enter();
+  if (p.deep != nullptr && pass == 2 && *p.deep == 0u) return;
   const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (j >= p.E) return;
@@ -182,7 +189,11 @@ __global__ void qb_scan_kernel(QbParams p, int pass) {
     p.prefix[j] = pre;
     p.rank[j] = rank - below;
     if (pass == 3) p.target[j] = -margin_from_key(pre);
-    if (pass == 1 && p.match != nullptr) { p.match[j] = count; p.fill[j] = 0u; }
+    if ((pass == 1 || pass == 2) && p.match != nullptr) {
+      p.match[j] = count;
+      p.fill[j] = 0u;
+      if (pass == 1 && p.deep != nullptr && count > (uint32_t)kQbListCap) atomicOr(p.deep, 1u);
+    }
   }
 }
 
@@ -196,6 +207,7 @@ __global__ void __launch_bounds__(kQbThreads) qb_gather_kernel(QbParams p) {
   const int col = blockIdx.x * kQbCols + lane;
   const bool live = col < p.E && p.match[col] <= (uint32_t)kQbListCap;
   const uint32_t pre = live ? p.prefix[col] : 0u;
+  const int fixed_shift = (*p.deep != 0u) ? 8 : 16;     // bits of the key not fixed yet
   const int rows_per = (p.m + gridDim.y - 1) / gridDim.y;
   const int r0 = blockIdx.y * rows_per;
   const int r1 = min(p.m, r0 + rows_per);
@@ -210,7 +222,7 @@ __global__ void __launch_bounds__(kQbThreads) qb_gather_kernel(QbParams p) {
 #pragma unroll
     for (int u = 0; u < kQbRowsInFlight; ++u) {
       const int i = i0 + u * kWarps;
-      if (live && i < r1 && ((key[u] ^ pre) >> 16) == 0u) {
+      if (live && i < r1 && ((key[u] ^ pre) >> fixed_shift) == 0u) {
         const uint32_t pos = atomicAdd(&p.fill[col], 1u);
         if (pos < (uint32_t)kQbListCap) p.list[(size_t)col * kQbListCap + pos] = (uint16_t)(key[u] & 0xffffu);
       }
@@ -234,18 +246,20 @@ __global__ void __launch_bounds__(kQbSelectWarps * 32) qb_select_kernel(QbParams
   const uint32_t n_match = p.match[j];
   const bool listed = n_match <= (uint32_t)kQbListCap;
   const uint32_t n = listed ? n_match : (uint32_t)p.m;
-  uint32_t pre = p.prefix[j];          // top 16 bits fixed
+  const bool deep = *p.deep != 0u;
+  const int fixed_shift = deep ? 8 : 16;
+  uint32_t pre = p.prefix[j];          // top 16 (24 after a third digit pass) bits fixed
   uint32_t rank = p.rank[j];           // 1-based rank inside the matching set
   const uint16_t* lst = p.list + (size_t)j * kQbListCap;
   auto value = [&](uint32_t i, bool& match) -> uint32_t {
     // low 16 bits of candidate i and whether it belongs to the matching set at all
     if (listed) { match = true; return (uint32_t)lst[i]; }
     const uint32_t key = __ldg(p.keys + (size_t)i * p.E + j);
-    match = ((key ^ pre) >> 16) == 0u;
+    match = ((key ^ pre) >> fixed_shift) == 0u;
     return key & 0xffffu;
   };
 #pragma unroll 1
-  for (int digit = 0; digit < 2; ++digit) {
+  for (int digit = deep ? 1 : 0; digit < 2; ++digit) {
     const int shift = 8 - 8 * digit;
 #pragma unroll
     for (int t = 0; t < 8; ++t) h[lane * 8 + t] = 0u;

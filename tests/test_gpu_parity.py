@@ -387,6 +387,44 @@ def test_quantile_controller_at_full_single_layer_size(K):
     assert 0 <= hist[0][0] <= wl.E / K - 1 + 1e-4
 
 
+def test_quantile_target_with_a_large_common_bias_offset():
+    # Quantile Balancing is not centred, so its bias drifts as a whole; with every bias near -1.5 the margins lie
+    # in [1, 2): sign, exponent and leading mantissa bits are common, and the keys that share the 16-bit prefix of
+    # an expert's quantile are far more than the 1024 a list holds.  The selection then takes a third digit pass;
+    # target and bias must still be those of the oracle's sort, bit for bit.
+    wl = synth.WORKLOADS["top3_single"].with_(H=512)
+    dev = "cuda"
+    g = torch.Generator().manual_seed(3)
+    b0 = (-1.5 + 0.002 * torch.randn(1, wl.E, generator=g)).float()
+    r = binding.Router(1, wl.E, wl.K, wl.H, wl.T, controller="quantile")
+    r.state_import(bias=b0.to(dev).contiguous())
+    w = torch.stack([synth.router_weights(wl, 0, dev)])
+    x = (torch.stack([synth.hidden_states(wl, 0, 0, dev)]).float() * 0.02).to(torch.bfloat16)   # scores close together
+    logits = torch.empty(1, wl.T, wl.E, device=dev)
+    alpha = torch.empty(1, wl.T, device=dev)
+    idx, gate = r.route_step(x, w, logits_out=logits, alpha_out=alpha)
+    r.controller_update()
+    r.poll()
+    loads, bias, _, _ = [np_(v) for v in r.load_stats()]
+    lg, al = np_(logits)[0], np_(alpha)[0]
+    oi = check_exact(lg, np_(b0)[0], wl.K, np_(idx)[0], np_(gate)[0], al)
+    np.testing.assert_array_equal(loads[0], np.bincount(oi.ravel(), minlength=wl.E))
+    Q = oracle.quantile_target(lg, al, wl.K)
+    want, _, _, _, _ = oracle_controller_step("quantile", np_(b0)[0], np.zeros(wl.E, np.float32), loads[0], dict(rho=0.0), False, Q)
+    np.testing.assert_array_equal(bits(bias[0]), bits(want))
+    # the premise: for some expert more than 1024 margins share the 16-bit key prefix of its quantile
+    d = (oracle.sigmoid_f32(lg[:, :8]) - al[:, None]).astype(np.float32)
+    u = (d + np.float32(0.0)).view(np.uint32)
+    keys = np.where(u & 0x80000000, ~u, u | 0x80000000).astype(np.uint32)
+    rank = wl.T - (wl.T * wl.K) // wl.E
+    most = 0
+    for j in range(8):
+        ans = np.sort(keys[:, j])[rank - 1]
+        most = max(most, int(((keys[:, j] >> 16) == (ans >> 16)).sum()))
+        assert np.float32(-(d[:, j][np.argsort(keys[:, j], kind="stable")[rank - 1]])) == Q[j]
+    assert most > 1024, most
+
+
 @pytest.mark.parametrize("bins,value_range,T,L", [(1024, 1.0, 3000, 1), (64, 0.5, 700, 2), (2048, 2.0, 16384, 1)])
 def test_quantile_controller_with_margin_histogram_estimate(bins, value_range, T, L):
     # footnote to Eq. 7: the target estimated from a per-expert margin histogram (this library's bin rule).
