@@ -106,7 +106,9 @@ typedef struct {
                            interpolation inside the bin that holds the r-th smallest margin:
                            estimate = -range + (k + ((r - below) - 0.5) / count_k) * (2 range / B).
                            |estimate - exact| < 2 range / B while the exact value is inside the range. */
-  float qb_hist_range;  /* > 0; default 1 */
+  float qb_hist_range;  /* > 0; default 1.  The margins of an expert are centred at minus the common part of the
+                           bias: an uncentred Quantile Balancing bias drifts as a whole, so choose centre = 1 or a
+                           range that covers the drift, or every margin ends up in an end bin */
 } moe_route_config;
 
 /* Fills *cfg with the paper's defaults (Ki = Kd = 6e-3, eta = 1e-3, rho = 0,
