@@ -640,10 +640,13 @@ def main():
             o_est = oj.prewarm(0.2, 3)
             o_steps = max(3, args.steps)
             o_rep = max(1, math.ceil(args.min_region_s * 1e3 / max(1e-6, o_est * o_steps)))
+            o_sampler = ClockSampler(local_rank)
+            o_sampler.start()
             o_ms, o_route, _ = oj.timed(o_steps, o_rep)
             while o_ms < args.min_region_s * 1e3:
                 o_rep = max(o_rep + 1, math.ceil(1.1 * o_rep * args.min_region_s * 1e3 / o_ms))
                 o_ms, o_route, _ = oj.timed(o_steps, o_rep)
+            o_clocks = o_sampler.stop()
             oj.router.poll()
             if dist is not None:
                 t = torch.tensor([o_ms], device=dev, dtype=torch.float64)
@@ -657,7 +660,8 @@ def main():
                                "tokens_per_s": o.L * o.T * world * o_steps * o_rep / (o_ms * 1e-3),
                                "tflops": rf["achieved"], "frac_of_burst": rf["frac_of_burst"],
                                "frac_of_sustained": rf["frac_of_sustained"], "ring": oj.ring,
-                               "traffic": rf["traffic"]})
+                               "traffic": rf["traffic"], "sm_mhz": o_clocks.get("sm_mhz"),
+                               "power_w": o_clocks.get("power_w"), "clock_reasons": o_clocks.get("reasons")})
             del oj
             torch.cuda.empty_cache()
 
