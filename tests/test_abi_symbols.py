@@ -52,6 +52,17 @@ def test_workspace_bytes_and_config_validation(lib):
     cq = binding.default_config(48, 768, 10, 2048, 16384)
     cq.controller = binding.MOE_CTRL_QUANTILE
     assert lib.moe_route_workspace_bytes(C.byref(cq)) >= n + 16384 * 768 * 4 + 768 * 256 * 4
+    # chunk-split scheduling reserves the per-chunk candidate lists; left to the library it is chosen for long
+    # hidden sizes and for launches with at most 64 (tile pair, chunk) items, and not otherwise
+    def ws(L, T, H, split):
+        c = binding.default_config(L, 768, 10, H, T)
+        c.chunk_split = split
+        return lib.moe_route_workspace_bytes(C.byref(c))
+    lists = lambda L, T: L * 3 * T * 11 * 8
+    assert ws(1, 1024, 256, 2) >= ws(1, 1024, 256, 1) + lists(1, 1024)
+    assert ws(1, 1024, 256, 0) == ws(1, 1024, 256, 2)            # 4 tile pairs x 3 chunks
+    assert ws(1, 16384, 2048, 0) == ws(1, 16384, 2048, 1)        # 64 tile pairs x 3 chunks, hidden 2048
+    assert ws(2, 4096, 4096, 0) == ws(2, 4096, 4096, 2)          # hidden 4096
     h = C.c_void_p()
     c = binding.default_config(1, 768, 10, 2048, 128)
     assert lib.moe_route_init(C.byref(c), None, 0, C.byref(h)) == binding.MOE_ERR_WORKSPACE
