@@ -9,6 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(HERE, "csrc", "moe_route.cu")
 LIB = os.path.join(HERE, "libmoe_route_b200.so")
 LIB_DEBUG = os.path.join(HERE, "libmoe_route_b200_debug.so")   # -DMOE_DEBUG: index guards + workspace canaries
+LIB_TIMERS = os.path.join(HERE, "libmoe_route_b200_timers.so")  # -DMOE_KERNEL_TIMERS: cycle accounting per warp role
 
 
 def sources():
@@ -25,14 +26,16 @@ def up_to_date(lib: str = LIB) -> bool:
     return all(os.path.getmtime(s) <= t for s in sources())
 
 
-def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
-    lib = LIB_DEBUG if debug else LIB
+def build(force: bool = False, verbose: bool = False, debug: bool = False, timers: bool = False) -> str:
+    lib = LIB_TIMERS if timers else LIB_DEBUG if debug else LIB
     if not force and up_to_date(lib):
         return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-fmad=false", "-shared", "-Xcompiler", "-fPIC", "-o", lib, SRC]
-    if debug:
+    if timers:
+        cmd.insert(1, "-DMOE_KERNEL_TIMERS")
+    elif debug:
         cmd.insert(1, "-DMOE_DEBUG")
     if verbose:
         cmd[1:1] = ["-Xptxas", "-v"]
@@ -45,4 +48,4 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv, timers="--timers" in sys.argv))
